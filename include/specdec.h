@@ -1,0 +1,175 @@
+/*
+ * specdec.h -- C ABI of the SpecDec++ verify/correct + adaptive-stop library (sm_100a).
+ *
+ * Operations follow arXiv 2405.19715:
+ *   - verify/correct: Algorithm 2 and the lower half of Algorithm 1 (accept test
+ *     r_i < p_i(y_i)/q_i(y_i), first rejection n, residual draw from Norm[(p-q)_+],
+ *     bonus draw from p_{K+1}); the rejection step itself is Appendix C.
+ *   - acceptance head: Eq. 3, sigmoid(f_theta(e_i)), with f_theta the (D+1)-layer
+ *     SiLU ResNet of Section 5.1.
+ *   - stop rule: Section 4.3 and the loop of Algorithm 1 (stop when
+ *     1 - prod_i sigmoid(f_theta(e_i)) > h).
+ *
+ * Conventions
+ *   - Every pointer marked "dev" is device memory of the context's GPU, owned by the
+ *     caller, neither retained nor freed by the library.  "host" pointers are ordinary
+ *     (preferably pinned) host memory.
+ *   - Tensors are dense row-major with the last index fastest.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream) unless stated otherwise; outputs are valid once the
+ *     stream has been synchronised.
+ *   - A context owns small scratch buffers.  Two calls that use the same context must
+ *     not overlap on the GPU (use one context per stream).
+ *   - Return value: SPECDEC_OK or an error code; specdec_last_error() gives a message.
+ *     Problems that only the device can see (a token outside [0,V), a length outside
+ *     [0,K]) never trap: the row's outputs become -1 and a sticky status word is set,
+ *     to be read with specdec_device_status().
+ */
+#ifndef SPECDEC_H_
+#define SPECDEC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct specdec_ctx specdec_ctx;
+
+typedef enum { SPECDEC_F32 = 0, SPECDEC_BF16 = 1 } specdec_dtype;
+
+typedef enum {
+    SPECDEC_OK = 0,
+    SPECDEC_EINVAL = 1,       /* bad host-visible argument                              */
+    SPECDEC_EUNSUPPORTED = 2, /* shape exceeds what the context / kernels were sized for */
+    SPECDEC_ECUDA = 3,        /* a CUDA runtime call failed                              */
+    SPECDEC_EDATA = 4         /* the device met a bad token or candidate length          */
+} specdec_status;
+
+/* Bits of the device status word returned by specdec_device_status(). */
+#define SPECDEC_DATA_BAD_LENGTH 1u /* some cand_len[b] outside [0,K]                     */
+#define SPECDEC_DATA_BAD_TOKEN  2u /* some cand_tokens[b,i] outside [0,V)                */
+#define SPECDEC_DATA_WAIT_LIMIT 4u /* a bounded in-kernel wait gave up (outputs invalid) */
+
+/* Kernel selection for specdec_verify_correct (flags argument). 0 lets the library pick. */
+#define SPECDEC_VERIFY_AUTO    0u
+#define SPECDEC_VERIFY_DIRECT  1u /* one CTA per (row, position), plain global loads      */
+#define SPECDEC_VERIFY_STREAM  2u /* persistent CTAs fed by bulk async copies (TMA)       */
+
+/*
+ * Create a context on `device` able to serve calls with B <= max_B and K <= max_K.
+ * Allocates the scratch used by verify/correct (per-(row,position) flags and draws,
+ * per-row arrival counters) and, when max_d > 0, the activation buffers of the
+ * acceptance head for max_B*max_K tokens of width max_d.  Ownership of *out passes to
+ * the caller (release with specdec_destroy).  Errors: EINVAL (null/negative), ECUDA.
+ */
+int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_d);
+int specdec_destroy(specdec_ctx* ctx);
+
+/* Message of the last error returned for this context (never NULL). */
+const char* specdec_last_error(const specdec_ctx* ctx);
+
+/*
+ * Synchronise `stream`, read and clear the sticky device status word.  *bits receives the
+ * SPECDEC_DATA_* bits (may be NULL).  Returns SPECDEC_OK if no bit was set, else SPECDEC_EDATA.
+ */
+int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits);
+
+/* Number of kernels this context has launched so far (for launch accounting). */
+uint64_t specdec_launch_count(const specdec_ctx* ctx);
+
+/*
+ * Verify and correct one speculation round for B independent rows
+ * (Algorithm 2; Algorithm 1 after its drafting loop; rejection step of Appendix C).
+ *
+ *   target_logits dev [B, K+1, V]  logits of the target model; row i scores position i,
+ *                                  row cand_len[b] is the "p_{K+1}" row of sequence b
+ *   draft_logits  dev [B, K, V]    logits of the draft model
+ *   dtype                          element type of both logit tensors
+ *   cand_tokens   dev [B, K] int32 drafted tokens y_i; entries at i >= cand_len[b] ignored
+ *   cand_len      dev [B] int32    candidates per row, 0 <= L <= K; NULL means L = K
+ *   uniforms      dev [B, K+1] f32 [b,i<K] = r_i of the accept test, [b,K] = the uniform
+ *                                  that draws y' (one fixed slot whatever cand_len[b] is)
+ *   temperature                    both models' logits are divided by it; must be > 0
+ *   n_accepted    dev out [B] int32  n = min({i < L : r_i >= p_i(y_i)/q_i(y_i)} U {L})
+ *   next_token    dev out [B] int32  y': inverse-CDF draw (vocabulary order, smallest j with
+ *                                  sum_{v<=j} w_v > u * sum_v w_v) from w = (p_n - q_n)_+ if
+ *                                  n < L, from w = p_L otherwise
+ *   accept_ratio  dev out [B, K] f32 or NULL: min(1, p_i(y_i)/q_i(y_i)) for i < L, 0 beyond
+ *   row_stats     dev out [B, K+1, 4] f32 (16-byte aligned) or NULL:
+ *                                  {lse_p, lse_q, p_i(y_i), q_i(y_i)} with
+ *                                  lse = log sum_v exp(logit_v / T); the bonus position L
+ *                                  holds {lse_p, 0, 0, 0}; positions > L hold zeros
+ *   resid_mass    dev out [B] f32 or NULL: sum_v (p_n - q_n)_+ at the first rejection,
+ *                                  1 when every candidate was accepted
+ *   flags                          SPECDEC_VERIFY_* kernel selection (0 = automatic)
+ *
+ * Logit rows at positions the method does not need (i > cand_len[b] of the target,
+ * i >= cand_len[b] of the draft) are never read.  Arithmetic is fp32 (exponentials by
+ * ex2.approx), the inverse-CDF prefix above 256-element slabs is accumulated in fp64.
+ * Errors: EINVAL (null pointer, B/K/V < 1, temperature <= 0 or not finite, unknown
+ * dtype/flags), EUNSUPPORTED (B or K beyond the context, V > 2^22, STREAM kernel
+ * requested for rows that are not 16-byte aligned), ECUDA.
+ */
+int specdec_verify_correct(specdec_ctx* ctx,
+                           const void* target_logits, const void* draft_logits, specdec_dtype dtype,
+                           const int32_t* cand_tokens, const int32_t* cand_len,
+                           const float* uniforms, float temperature,
+                           int B, int K, int V,
+                           int32_t* n_accepted, int32_t* next_token,
+                           float* accept_ratio, float* row_stats, float* resid_mass,
+                           uint32_t flags, void* stream);
+
+/*
+ * Same operation with HOST input and output buffers: copies the inputs to device staging
+ * buffers owned by the context (allocated or grown on first use), runs the kernels, copies
+ * n_accepted / next_token (and accept_ratio when not NULL) back and synchronises `stream`
+ * before returning.  Pinned host memory lets the copies run at full PCIe rate.
+ */
+int specdec_verify_correct_host(specdec_ctx* ctx,
+                                const void* target_logits, const void* draft_logits, specdec_dtype dtype,
+                                const int32_t* cand_tokens, const int32_t* cand_len,
+                                const float* uniforms, float temperature,
+                                int B, int K, int V,
+                                int32_t* n_accepted, int32_t* next_token, float* accept_ratio,
+                                uint32_t flags, void* stream);
+
+/*
+ * Acceptance-prediction head (Eq. 3; architecture of Section 5.1):
+ *   x_0 = hidden;  x_k = x_{k-1} + SiLU(W_k x_{k-1} + b_k), k = 1..depth;
+ *   accept_prob = sigmoid(w_out . x_depth + b_out).
+ * All tensors bf16 on the device; W_k is [d, d] stored (out, in) like a linear layer's
+ * weight; b_k [d] may be NULL (zero).  GEMMs run on tcgen05 tensor cores with fp32
+ * accumulation; activations between blocks are rounded to bf16.
+ */
+typedef struct {
+    const void* const* W;   /* host array of `depth` dev pointers, each bf16 [d, d]        */
+    const void* const* b;   /* host array of `depth` dev pointers (bf16 [d]) or NULL entries; may be NULL */
+    const void* w_out;      /* dev bf16 [d]                                                */
+    float b_out;
+    int d;                  /* hidden width, multiple of 128                               */
+    int depth;              /* number of residual blocks D, 0 <= D <= 8                    */
+} specdec_head;
+
+/*
+ *   hidden      dev [B, K, d] bf16   final hidden state e_i of each drafted token
+ *   accept_prob dev out [B, K] f32   sigmoid(f_theta(e_i))
+ * Errors: EINVAL, EUNSUPPORTED (d not a multiple of 128, B*K or d beyond the context), ECUDA.
+ */
+int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const specdec_head* head,
+                        int B, int K, float* accept_prob, void* stream);
+
+/*
+ * Threshold stop rule (Section 4.3; loop of Algorithm 1): for each row the first 0-based
+ * position j with 1 - prod_{i<=j} accept_prob[b,i] > h (strict), scanning i < cand_len[b]
+ * (K when cand_len is NULL).  stop_pos[b] = j, or cand_len[b] (resp. K) if the rule never
+ * fires.  Products are formed sequentially in fp32.
+ *   accept_prob dev [B, K] f32, cand_len dev [B] int32 or NULL, stop_pos dev out [B] int32
+ */
+int specdec_stop(specdec_ctx* ctx, const float* accept_prob, const int32_t* cand_len,
+                 float h, int B, int K, int32_t* stop_pos, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECDEC_H_ */

@@ -1,0 +1,241 @@
+// C ABI of libspecdec: context management, argument checks and dispatch to the launchers.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "specdec_internal.h"
+
+namespace {
+
+int fail(specdec_ctx* ctx, int code, const char* fmt, ...) {
+    if (ctx) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(ctx->err, sizeof(ctx->err), fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+int cuda_fail(specdec_ctx* ctx, cudaError_t e, const char* what) {
+    return fail(ctx, SPECDEC_ECUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define CU(ctx, call)                                              \
+    do {                                                           \
+        cudaError_t e__ = (call);                                  \
+        if (e__ != cudaSuccess) return cuda_fail(ctx, e__, #call); \
+    } while (0)
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int check_verify_args(specdec_ctx* ctx, const void* target, const void* draft, int dtype, const int32_t* tokens,
+                      const float* uniforms, float T, int B, int K, int V, const int32_t* n_acc,
+                      const int32_t* next, uint32_t flags) {
+    if (!ctx) return SPECDEC_EINVAL;
+    if (!target || !draft || !tokens || !uniforms || !n_acc || !next)
+        return fail(ctx, SPECDEC_EINVAL, "verify_correct: null pointer argument");
+    if (dtype != SPECDEC_F32 && dtype != SPECDEC_BF16) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown dtype %d", dtype);
+    if (B < 1 || K < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "verify_correct: B, K, V must be >= 1 (got %d, %d, %d)", B, K, V);
+    if (!(T > 0.f) || !std::isfinite(T)) return fail(ctx, SPECDEC_EINVAL, "verify_correct: temperature must be positive and finite");
+    if (flags > SPECDEC_VERIFY_STREAM) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown flags %u", flags);
+    if (B > ctx->max_B || K > ctx->max_K)
+        return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: B=%d K=%d exceed the context (max_B=%d max_K=%d)", B, K, ctx->max_B, ctx->max_K);
+    if (V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: V=%d above 2^22", V);
+    return SPECDEC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_d) {
+    if (!out || max_B < 1 || max_K < 1 || max_d < 0 || device < 0) return SPECDEC_EINVAL;
+    *out = nullptr;
+    if ((long long)max_B * (max_K + 1) > (1ll << 28)) return SPECDEC_EINVAL;
+    specdec_ctx* ctx = new (std::nothrow) specdec_ctx();
+    if (!ctx) return SPECDEC_ECUDA;
+    ctx->device = device;
+    ctx->max_B = max_B;
+    ctx->max_K = max_K;
+    ctx->max_d = max_d;
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    const size_t nflag = (size_t)max_B * max_K, ndraw = (size_t)max_B * (max_K + 1);
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->flags, nflag * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->draws, ndraw * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->draw_mass, ndraw * sizeof(float));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->arrive, (size_t)max_B * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->status, sizeof(uint32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->flags, 0, nflag * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->arrive, 0, (size_t)max_B * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
+    if (e == cudaSuccess && max_d > 0) {
+        const size_t act = (size_t)max_B * max_K * max_d * 2;
+        e = cudaMalloc(&ctx->act[0], act);
+        if (e == cudaSuccess) e = cudaMalloc(&ctx->act[1], act);
+        if (e == cudaSuccess)
+            e = cudaMalloc(&ctx->head_partial, (size_t)max_B * max_K * ((max_d + 127) / 128) * sizeof(float));
+    }
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        specdec_destroy(ctx);
+        return SPECDEC_ECUDA;
+    }
+    *out = ctx;
+    return SPECDEC_OK;
+}
+
+int specdec_destroy(specdec_ctx* ctx) {
+    if (!ctx) return SPECDEC_EINVAL;
+    cudaSetDevice(ctx->device);
+    cudaFree(ctx->flags);
+    cudaFree(ctx->draws);
+    cudaFree(ctx->draw_mass);
+    cudaFree(ctx->arrive);
+    cudaFree(ctx->status);
+    cudaFree(ctx->stage);
+    cudaFree(ctx->act[0]);
+    cudaFree(ctx->act[1]);
+    cudaFree(ctx->head_partial);
+    delete ctx;
+    return SPECDEC_OK;
+}
+
+const char* specdec_last_error(const specdec_ctx* ctx) { return ctx ? ctx->err : "null context"; }
+
+uint64_t specdec_launch_count(const specdec_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits) {
+    if (!ctx) return SPECDEC_EINVAL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint32_t host = 0;
+    CU(ctx, cudaMemcpyAsync(&host, ctx->status, sizeof(host), cudaMemcpyDeviceToHost, s));
+    CU(ctx, cudaMemsetAsync(ctx->status, 0, sizeof(uint32_t), s));
+    CU(ctx, cudaStreamSynchronize(s));
+    if (bits) *bits = host;
+    if (host) return fail(ctx, SPECDEC_EDATA, "device status bits 0x%x (1 = bad cand_len, 2 = bad token, 4 = wait limit)", host);
+    return SPECDEC_OK;
+}
+
+int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const void* draft_logits,
+                           specdec_dtype dtype, const int32_t* cand_tokens, const int32_t* cand_len,
+                           const float* uniforms, float temperature, int B, int K, int V, int32_t* n_accepted,
+                           int32_t* next_token, float* accept_ratio, float* row_stats, float* resid_mass,
+                           uint32_t flags, void* stream) {
+    int rc = check_verify_args(ctx, target_logits, draft_logits, (int)dtype, cand_tokens, uniforms, temperature, B,
+                               K, V, n_accepted, next_token, flags);
+    if (rc != SPECDEC_OK) return rc;
+    if (row_stats && reinterpret_cast<uintptr_t>(row_stats) % 16 != 0)
+        return fail(ctx, SPECDEC_EINVAL, "verify_correct: row_stats must be 16-byte aligned");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    ctx->epoch = (ctx->epoch + 1) & 0x3fffffffu;
+    if (ctx->epoch == 0) {   // wrapped: forget every stale flag before reusing epoch numbers
+        CU(ctx, cudaMemsetAsync(ctx->flags, 0, (size_t)ctx->max_B * ctx->max_K * sizeof(int32_t), s));
+        ctx->epoch = 1;
+    }
+    VerifyParams p;
+    p.target = target_logits;
+    p.draft = draft_logits;
+    p.tokens = cand_tokens;
+    p.lens = cand_len;
+    p.uniforms = uniforms;
+    p.c = (float)(1.4426950408889634 / (double)temperature);
+    p.B = B;
+    p.K = K;
+    p.V = V;
+    p.n_acc = n_accepted;
+    p.next = next_token;
+    p.ratio = accept_ratio;
+    p.stats = row_stats;
+    p.rmass = resid_mass;
+    p.flags = ctx->flags;
+    p.draws = ctx->draws;
+    p.draw_mass = ctx->draw_mass;
+    p.arrive = ctx->arrive;
+    p.status = ctx->status;
+    p.epoch = ctx->epoch;
+
+    const bool stream_ok = verify_stream_supported(p, dtype);
+    bool use_stream;
+    if (flags == SPECDEC_VERIFY_STREAM) {
+        if (!stream_ok)
+            return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: streaming kernel needs 16-byte aligned rows (V=%d)", V);
+        use_stream = true;
+    } else if (flags == SPECDEC_VERIFY_DIRECT) {
+        use_stream = false;
+    } else {
+        use_stream = stream_ok;
+    }
+    int n_launch = 0;
+    cudaError_t e = use_stream ? launch_verify_stream(p, dtype, ctx->sm_count, s, &n_launch)
+                               : launch_verify_direct(p, dtype, s, &n_launch);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "verify_correct launch");
+    ctx->launches += n_launch;
+    return SPECDEC_OK;
+}
+
+int specdec_verify_correct_host(specdec_ctx* ctx, const void* target_logits, const void* draft_logits,
+                                specdec_dtype dtype, const int32_t* cand_tokens, const int32_t* cand_len,
+                                const float* uniforms, float temperature, int B, int K, int V,
+                                int32_t* n_accepted, int32_t* next_token, float* accept_ratio, uint32_t flags,
+                                void* stream) {
+    int rc = check_verify_args(ctx, target_logits, draft_logits, (int)dtype, cand_tokens, uniforms, temperature, B,
+                               K, V, n_accepted, next_token, flags);
+    if (rc != SPECDEC_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t es = dtype == SPECDEC_BF16 ? 2 : 4;
+    const size_t t_bytes = (size_t)B * (K + 1) * V * es, d_bytes = (size_t)B * K * V * es;
+    const size_t tok_bytes = (size_t)B * K * 4, len_bytes = (size_t)B * 4, uni_bytes = (size_t)B * (K + 1) * 4;
+    size_t off = 0;
+    const size_t o_t = off;   off = align_up(off + t_bytes, 256);
+    const size_t o_d = off;   off = align_up(off + d_bytes, 256);
+    const size_t o_tok = off; off = align_up(off + tok_bytes, 256);
+    const size_t o_len = off; off = align_up(off + len_bytes, 256);
+    const size_t o_uni = off; off = align_up(off + uni_bytes, 256);
+    const size_t o_n = off;   off = align_up(off + len_bytes, 256);
+    const size_t o_nx = off;  off = align_up(off + len_bytes, 256);
+    const size_t o_r = off;   off = align_up(off + tok_bytes, 256);
+    if (off > ctx->stage_bytes) {
+        CU(ctx, cudaStreamSynchronize(s));
+        cudaFree(ctx->stage);
+        ctx->stage = nullptr;
+        ctx->stage_bytes = 0;
+        CU(ctx, cudaMalloc(&ctx->stage, off));
+        ctx->stage_bytes = off;
+    }
+    char* base = static_cast<char*>(ctx->stage);
+    CU(ctx, cudaMemcpyAsync(base + o_t, target_logits, t_bytes, cudaMemcpyHostToDevice, s));
+    CU(ctx, cudaMemcpyAsync(base + o_d, draft_logits, d_bytes, cudaMemcpyHostToDevice, s));
+    CU(ctx, cudaMemcpyAsync(base + o_tok, cand_tokens, tok_bytes, cudaMemcpyHostToDevice, s));
+    if (cand_len) CU(ctx, cudaMemcpyAsync(base + o_len, cand_len, len_bytes, cudaMemcpyHostToDevice, s));
+    CU(ctx, cudaMemcpyAsync(base + o_uni, uniforms, uni_bytes, cudaMemcpyHostToDevice, s));
+    rc = specdec_verify_correct(ctx, base + o_t, base + o_d, dtype, reinterpret_cast<int32_t*>(base + o_tok),
+                                cand_len ? reinterpret_cast<int32_t*>(base + o_len) : nullptr,
+                                reinterpret_cast<float*>(base + o_uni), temperature, B, K, V,
+                                reinterpret_cast<int32_t*>(base + o_n), reinterpret_cast<int32_t*>(base + o_nx),
+                                accept_ratio ? reinterpret_cast<float*>(base + o_r) : nullptr, nullptr, nullptr,
+                                flags, s);
+    if (rc != SPECDEC_OK) return rc;
+    CU(ctx, cudaMemcpyAsync(n_accepted, base + o_n, len_bytes, cudaMemcpyDeviceToHost, s));
+    CU(ctx, cudaMemcpyAsync(next_token, base + o_nx, len_bytes, cudaMemcpyDeviceToHost, s));
+    if (accept_ratio) CU(ctx, cudaMemcpyAsync(accept_ratio, base + o_r, tok_bytes, cudaMemcpyDeviceToHost, s));
+    CU(ctx, cudaStreamSynchronize(s));
+    return SPECDEC_OK;
+}
+
+int specdec_stop(specdec_ctx* ctx, const float* accept_prob, const int32_t* cand_len, float h, int B, int K,
+                 int32_t* stop_pos, void* stream) {
+    if (!ctx) return SPECDEC_EINVAL;
+    if (!accept_prob || !stop_pos) return fail(ctx, SPECDEC_EINVAL, "stop: null pointer argument");
+    if (B < 1 || K < 1) return fail(ctx, SPECDEC_EINVAL, "stop: B and K must be >= 1");
+    if (h != h) return fail(ctx, SPECDEC_EINVAL, "stop: threshold is NaN");
+    cudaError_t e = launch_stop(accept_prob, cand_len, h, B, K, stop_pos, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "stop launch");
+    ctx->launches += 1;
+    return SPECDEC_OK;
+}
+
+}  // extern "C"

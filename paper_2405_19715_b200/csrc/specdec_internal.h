@@ -1,0 +1,57 @@
+// Internal declarations shared by the translation units of libspecdec (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "specdec.h"
+
+struct specdec_ctx {
+    int device = 0;
+    int max_B = 0, max_K = 0, max_d = 0;
+    int sm_count = 0;
+    // verify/correct scratch (device)
+    int32_t* flags = nullptr;     // [max_B * max_K]      (epoch << 2) | state of each accept test
+    int32_t* draws = nullptr;     // [max_B * (max_K+1)]  candidate y' drawn at each position
+    float* draw_mass = nullptr;   // [max_B * (max_K+1)]  mass of the weights that draw came from
+    int32_t* arrive = nullptr;    // [max_B]              positions of a row that have finished
+    uint32_t* status = nullptr;   // sticky SPECDEC_DATA_* bits
+    uint32_t epoch = 0;
+    uint64_t launches = 0;
+    // staging for the host-buffer entry point (device), grown on demand
+    void* stage = nullptr;
+    size_t stage_bytes = 0;
+    // acceptance-head activations (device, bf16) and split-N partial logits
+    void* act[2] = {nullptr, nullptr};   // [max_B*max_K, max_d] each
+    float* head_partial = nullptr;       // [max_B*max_K, max_d/128]
+    char err[256] = "no error";
+};
+
+struct VerifyParams {
+    const void* target;
+    const void* draft;
+    const int32_t* tokens;
+    const int32_t* lens;
+    const float* uniforms;
+    float c;              // log2(e) / T: logits are scaled into base-2 exponents
+    int B, K, V;
+    int32_t* n_acc;
+    int32_t* next;
+    float* ratio;
+    float* stats;
+    float* rmass;
+    int32_t* flags;
+    int32_t* draws;
+    float* draw_mass;
+    int32_t* arrive;
+    uint32_t* status;
+    uint32_t epoch;
+};
+
+// Launchers (verify.cu, verify_stream.cu, stop.cu, head.cu).  Return a cudaError_t.
+cudaError_t launch_verify_direct(const VerifyParams& p, specdec_dtype dtype, cudaStream_t s, int* n_launch);
+cudaError_t launch_verify_stream(const VerifyParams& p, specdec_dtype dtype, int sm_count, cudaStream_t s,
+                                 int* n_launch);
+bool verify_stream_supported(const VerifyParams& p, specdec_dtype dtype);
+cudaError_t launch_stop(const float* accept_prob, const int32_t* lens, float h, int B, int K,
+                        int32_t* stop_pos, cudaStream_t s);

@@ -1,0 +1,30 @@
+// Threshold stop rule (Section 4.3 and the loop of Algorithm 1, arXiv 2405.19715):
+// p_hat <- p_hat * accept_prob[i]; stop at the first i with 1 - p_hat > h.
+#include "specdec_internal.h"
+
+namespace {
+
+__global__ void stop_kernel(const float* __restrict__ a, const int32_t* __restrict__ lens, float h, int B, int K,
+                            int32_t* __restrict__ stop_pos) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    int L = lens ? lens[b] : K;
+    L = L < 0 ? 0 : (L > K ? K : L);
+    const float* row = a + (size_t)b * K;
+    float c = 1.f;
+    int pos = L;
+    for (int j = 0; j < L; ++j) {
+        c *= row[j];
+        if (1.f - c > h) { pos = j; break; }
+    }
+    stop_pos[b] = pos;
+}
+
+}  // namespace
+
+cudaError_t launch_stop(const float* accept_prob, const int32_t* lens, float h, int B, int K, int32_t* stop_pos,
+                        cudaStream_t s) {
+    const int threads = 128;
+    stop_kernel<<<(B + threads - 1) / threads, threads, 0, s>>>(accept_prob, lens, h, B, K, stop_pos);
+    return cudaGetLastError();
+}

@@ -1,0 +1,376 @@
+// Device-side building blocks of verify/correct (Algorithm 2 of arXiv 2405.19715):
+// softmax statistics with a lazily re-referenced running sum, the accept test, the
+// residual / bonus inverse-CDF draw and the per-row first-rejection ballot.
+// Used by the direct kernel (verify.cu) and the streaming kernel (verify_stream.cu).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "specdec_internal.h"
+
+namespace sd {
+
+constexpr float NEG_BIG = -1.0e30f;      // "no reference yet": any finite logit re-references
+constexpr int FLAG_ACCEPT = 1, FLAG_REJECT = 2, FLAG_BAD = 3;
+
+template <typename T> struct Elem;
+template <> struct Elem<float> { static constexpr int EPV = 4; };           // elements per 16 bytes
+template <> struct Elem<__nv_bfloat16> { static constexpr int EPV = 8; };
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ int ld_acquire(const int32_t* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_release(int32_t* p, int v) {
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void bar_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+__device__ __forceinline__ void unpack(const uint4& r, float (&x)[4]) {
+    x[0] = __uint_as_float(r.x); x[1] = __uint_as_float(r.y);
+    x[2] = __uint_as_float(r.z); x[3] = __uint_as_float(r.w);
+}
+__device__ __forceinline__ void unpack(const uint4& r, float (&x)[8]) {   // 8 bf16 -> fp32, exact
+    x[0] = __uint_as_float(r.x << 16); x[1] = __uint_as_float(r.x & 0xffff0000u);
+    x[2] = __uint_as_float(r.y << 16); x[3] = __uint_as_float(r.y & 0xffff0000u);
+    x[4] = __uint_as_float(r.z << 16); x[5] = __uint_as_float(r.z & 0xffff0000u);
+    x[6] = __uint_as_float(r.w << 16); x[7] = __uint_as_float(r.w & 0xffff0000u);
+}
+
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// Vector j (EPV consecutive elements) of a row.  VEC: one 16-byte load through L2 only.
+// Otherwise element loads with everything at or beyond V read as -inf (weight zero).
+template <typename T, bool VEC>
+__device__ __forceinline__ void load_vec(const T* __restrict__ row, int j, int V, float (&x)[Elem<T>::EPV]) {
+    constexpr int N = Elem<T>::EPV;
+    if constexpr (VEC) {
+        uint4 r = __ldcg(reinterpret_cast<const uint4*>(row) + j);
+        unpack(r, x);
+    } else {
+        const int v0 = j * N;
+#pragma unroll
+        for (int k = 0; k < N; ++k) x[k] = (v0 + k < V) ? to_float(row[v0 + k]) : -INFINITY;
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Running sum of 2^(x*c - rs).  The reference rs follows the data lazily: it is replaced by
+// the current vector's maximum only when that vector's terms sum above 256*N, i.e. when some
+// logit sits more than ~8 binades above the reference.  Exponent arguments of the terms that
+// matter therefore stay small (accurate), nothing can overflow, and the common case costs one
+// compare and one not-taken branch per vector instead of a maximum per element.
+struct Acc {
+    float rs, s;
+};
+__device__ __forceinline__ Acc acc_init() { return Acc{NEG_BIG, 0.f}; }
+
+template <int N>
+__device__ __forceinline__ float sum_tree(const float (&e)[N]) {
+    if constexpr (N == 8) return ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
+    else return (e[0] + e[1]) + (e[2] + e[3]);
+}
+
+template <int N>
+__device__ __forceinline__ void acc_update(Acc& a, const float (&x)[N], float c) {
+    float e[N];
+#pragma unroll
+    for (int k = 0; k < N; ++k) e[k] = ex2(fmaf(x[k], c, -a.rs));
+    float vs = sum_tree<N>(e);
+    if (!(vs <= 256.f * N)) {
+        float m = x[0];
+#pragma unroll
+        for (int k = 1; k < N; ++k) m = fmaxf(m, x[k]);
+        if (m >= -3.0e38f) {                       // a finite (or +inf) maximum: re-reference
+            const float nrs = m * c;
+            a.s *= ex2(a.rs - nrs);
+            a.rs = nrs;
+#pragma unroll
+            for (int k = 0; k < N; ++k) e[k] = ex2(fmaf(x[k], c, -nrs));
+            vs = sum_tree<N>(e);
+        } else {
+            vs = (m != m) ? m : 0.f;               // all NaN propagates; all -inf adds nothing
+        }
+    }
+    a.s += vs;
+}
+
+__device__ __forceinline__ Acc acc_merge(const Acc& a, const Acc& b) {
+    Acc r;
+    r.rs = fmaxf(a.rs, b.rs);
+    r.s = a.s * ex2(a.rs - r.rs) + b.s * ex2(b.rs - r.rs);
+    return r;
+}
+
+__device__ __forceinline__ Acc warp_merge(Acc a) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Acc b;
+        b.rs = __shfl_xor_sync(0xffffffffu, a.rs, o);
+        b.s = __shfl_xor_sync(0xffffffffu, a.s, o);
+        a = acc_merge(a, b);
+    }
+    return a;
+}
+
+// log2 of the normaliser as an unevaluated sum hi + lo (fp32 each) so that per-element
+// probabilities 2^(x*c - hi - lo) carry no common scale error.
+struct Norm {
+    float hi, lo;
+};
+__device__ __forceinline__ Norm make_norm(const Acc& a) {
+    const double k = (double)a.rs + log2((double)a.s);
+    Norm n;
+    n.hi = (float)k;
+    n.lo = (float)(k - (double)n.hi);
+    return n;
+}
+__device__ __forceinline__ float prob(float x, float c, const Norm& n) {
+    return ex2(fmaf(x, c, -n.hi) - n.lo);
+}
+
+// Shared-memory scratch of one CTA handling one (row, position) unit.
+struct UnitShared {
+    Acc wp[32], wq[32];        // per-warp partial statistics
+    Norm np, nq;               // normalisers of the unit
+    int need_draw;             // 0 none, 1 residual, 2 target itself
+    int token;
+    double total;
+};
+
+struct Unit {
+    int b, i, L;               // row, position, candidate length of the row
+    bool bonus;                // i == L: the p_{L+1} row, no draft
+};
+
+// Called by one thread once the unit's statistics are known: accept test, optional outputs,
+// flag publication and the decision whether this unit must produce a draw.
+__device__ __forceinline__ int unit_decide(const VerifyParams& P, const Unit& u, const Acc& ap, const Acc& aq,
+                                           float t_y, float d_y, int y_ok) {
+    const int K = P.K;
+    const float LN2 = 0.6931471805599453f;
+    int state = 0;
+    if (!u.bonus) {
+        // log2 p(y) and log2 q(y); the references cancel exactly because each term is formed
+        // against the same rs the sum was accumulated with.
+        const float lp = fmaf(t_y, P.c, -ap.rs) - log2f(ap.s);
+        const float lq = fmaf(d_y, P.c, -aq.rs) - log2f(aq.s);
+        const float ratio = exp2f(lp - lq);
+        const float r = P.uniforms[(size_t)u.b * (K + 1) + u.i];
+        state = !y_ok ? FLAG_BAD : (r >= ratio ? FLAG_REJECT : FLAG_ACCEPT);   // r == ratio rejects
+        if (!y_ok) atomicOr(P.status, SPECDEC_DATA_BAD_TOKEN);
+        if (P.ratio) P.ratio[(size_t)u.b * K + u.i] = y_ok ? fminf(1.f, ratio) : -1.f;
+        if (P.stats) {
+            float4 st;
+            st.x = (ap.rs + log2f(ap.s)) * LN2;
+            st.y = (aq.rs + log2f(aq.s)) * LN2;
+            st.z = exp2f(lp);
+            st.w = exp2f(lq);
+            reinterpret_cast<float4*>(P.stats)[(size_t)u.b * (K + 1) + u.i] = st;
+        }
+        st_release(&P.flags[(size_t)u.b * K + u.i], (int)((P.epoch << 2) | (uint32_t)state));
+    } else if (P.stats) {
+        float4 st = make_float4((ap.rs + log2f(ap.s)) * LN2, 0.f, 0.f, 0.f);
+        reinterpret_cast<float4*>(P.stats)[(size_t)u.b * (K + 1) + u.i] = st;
+    }
+    // A draw is needed only if this position can be the first rejection (or the bonus draw):
+    // skip it when an earlier position of the row is already known to have rejected.
+    bool known = false;
+    for (int j = 0; j < u.i; ++j) {
+        const int f = ld_acquire(&P.flags[(size_t)u.b * K + j]);
+        if (((uint32_t)f >> 2) == P.epoch && (f & 3) >= FLAG_REJECT) known = true;
+    }
+    if (known || state == FLAG_BAD) return 0;
+    if (u.bonus) return 2;
+    return state == FLAG_REJECT ? 1 : 0;
+}
+
+// Weights y' is drawn from, for one vector: (p - q)_+ (mode 1) or p (mode 2).
+template <int N>
+__device__ __forceinline__ float vec_weights(const float (&xt)[N], const float (&xd)[N], float c, const Norm& np,
+                                             const Norm& nq, int mode, float (&w)[N]) {
+    float sum = 0.f;
+#pragma unroll
+    for (int k = 0; k < N; ++k) {
+        const float p = prob(xt[k], c, np);
+        w[k] = (mode == 1) ? fmaxf(p - prob(xd[k], c, nq), 0.f) : p;
+        sum += w[k];
+    }
+    return sum;
+}
+
+// Block-wide inverse-CDF draw over the rows of one unit, read from global memory (L2).
+// A slab is the 32*EPV consecutive elements one warp covers with one vector per lane; slab
+// sums are fp32, everything above them is fp64.  Leaves the token in sh.token and the total
+// mass in sh.total.  All `nthreads` threads (tid 0..nthreads-1, whole warps) must call; uses
+// named barrier `bar_id`.
+template <typename T, bool VEC>
+__device__ void unit_draw(const VerifyParams& P, const T* __restrict__ trow, const T* __restrict__ drow, int mode,
+                          float u01, UnitShared& sh, float* __restrict__ slab_sum, int tid, int nthreads, int bar_id) {
+    constexpr int N = Elem<T>::EPV;
+    const int V = P.V;
+    const int nvec = (V + N - 1) / N;
+    const int nslab = (nvec + 31) / 32;
+    const int warp = tid >> 5, lane = tid & 31, nwarp = nthreads >> 5;
+    const Norm np = sh.np, nq = sh.nq;
+    float xt[N], xd[N], w[N];
+#pragma unroll
+    for (int k = 0; k < N; ++k) xd[k] = 0.f;
+
+    for (int s = warp; s < nslab; s += nwarp) {
+        const int j = s * 32 + lane;
+        float ls = 0.f;
+        if (j < nvec) {
+            load_vec<T, VEC>(trow, j, V, xt);
+            if (mode == 1) load_vec<T, VEC>(drow, j, V, xd);
+            ls = vec_weights<N>(xt, xd, P.c, np, nq, mode, w);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+        if (lane == 0) slab_sum[s] = ls;
+    }
+    bar_sync(bar_id, nthreads);
+
+    if (warp == 0) {
+        // fp64 prefix over slabs: each lane owns a contiguous run of slabs
+        const int per = (nslab + 31) / 32;
+        const int s0 = min(lane * per, nslab), s1 = min(s0 + per, nslab);
+        double mine = 0.0;
+        for (int s = s0; s < s1; ++s) mine += (double)slab_sum[s];
+        double incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        const double total = __shfl_sync(0xffffffffu, incl, 31);
+        const double tau = (double)u01 * total;
+        // first slab whose inclusive prefix exceeds tau
+        double run = incl - mine;
+        int found = -1;
+        double base = 0.0;
+        for (int s = s0; s < s1; ++s) {
+            const double nxt = run + (double)slab_sum[s];
+            if (found < 0 && nxt > tau) { found = s; base = run; }
+            run = nxt;
+        }
+        const unsigned m = __ballot_sync(0xffffffffu, found >= 0);
+        int slab;
+        if (m) {
+            const int src = __ffs(m) - 1;
+            slab = __shfl_sync(0xffffffffu, found, src);
+            base = __shfl_sync(0xffffffffu, base, src);
+        } else {
+            // rounding left nothing above tau: take the last slab with positive mass
+            int lastpos = -1;
+            double lb = 0.0;
+            run = incl - mine;
+            for (int s = s0; s < s1; ++s) {
+                if (slab_sum[s] > 0.f) { lastpos = s; lb = run; }
+                run += (double)slab_sum[s];
+            }
+            const unsigned pm = __ballot_sync(0xffffffffu, lastpos >= 0);
+            const int src = pm ? 31 - __clz(pm) : 0;
+            slab = __shfl_sync(0xffffffffu, lastpos, src);
+            base = __shfl_sync(0xffffffffu, lb, src);
+            if (slab < 0) { slab = 0; base = 0.0; }
+        }
+        // walk inside the slab
+        const int j = slab * 32 + lane;
+        float ls = 0.f;
+#pragma unroll
+        for (int k = 0; k < N; ++k) w[k] = 0.f;
+        if (j < nvec) {
+            load_vec<T, VEC>(trow, j, V, xt);
+            if (mode == 1) load_vec<T, VEC>(drow, j, V, xd);
+            ls = vec_weights<N>(xt, xd, P.c, np, nq, mode, w);
+        }
+        float li = ls;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float up = __shfl_up_sync(0xffffffffu, li, o);
+            if (lane >= o) li += up;
+        }
+        float lex = __shfl_up_sync(0xffffffffu, li, 1);
+        if (lane == 0) lex = 0.f;
+        const unsigned hm = __ballot_sync(0xffffffffu, base + (double)li > tau);
+        const unsigned pm = __ballot_sync(0xffffffffu, ls > 0.f);
+        const int sel = hm ? __ffs(hm) - 1 : (pm ? 31 - __clz(pm) : -1);
+        int tok = min(slab * 32 * N, V - 1);
+        if (sel >= 0 && lane == sel) {
+            double acc = base + (double)lex;
+            int pick = -1, lastp = 0;
+#pragma unroll
+            for (int k = 0; k < N; ++k) {
+                acc += (double)w[k];
+                if (w[k] > 0.f) lastp = k;
+                if (pick < 0 && acc > tau) pick = k;
+            }
+            if (pick < 0) pick = lastp;
+            tok = min(j * N + pick, V - 1);
+        }
+        if (sel >= 0) tok = __shfl_sync(0xffffffffu, tok, sel);
+        if (lane == 0) { sh.token = tok; sh.total = total; }
+    }
+    bar_sync(bar_id, nthreads);
+}
+
+// Row bookkeeping by one full warp of a unit after its (optional) draw: record the draw, count
+// the arrival, and let the last position of the row to arrive resolve n and y' (warp ballot
+// over the accept flags of positions < L).
+__device__ __forceinline__ void unit_finish(const VerifyParams& P, const Unit& u, int have_draw, int token, float mass,
+                                            int lane) {
+    const int K = P.K;
+    int last = 0;
+    if (lane == 0) {
+        P.draws[(size_t)u.b * (K + 1) + u.i] = have_draw ? token : -1;
+        P.draw_mass[(size_t)u.b * (K + 1) + u.i] = mass;
+        __threadfence();
+        const int old = atomicAdd(&P.arrive[u.b], 1);
+        last = (old == u.L);
+        if (last) __threadfence();
+    }
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (!last) return;
+    int n = u.L, bad = 0;
+    for (int j0 = 0; j0 < u.L; j0 += 32) {
+        const int j = j0 + lane;
+        int st = FLAG_ACCEPT;
+        if (j < u.L) st = ld_acquire(&P.flags[(size_t)u.b * K + j]) & 3;
+        const unsigned rej = __ballot_sync(0xffffffffu, st >= FLAG_REJECT);
+        const unsigned bd = __ballot_sync(0xffffffffu, st == FLAG_BAD);
+        if (rej && n == u.L) n = j0 + __ffs(rej) - 1;
+        bad |= (bd != 0);
+    }
+    if (lane == 0) {
+        int tok = -1;
+        float m = 0.f;
+        if (!bad) {
+            tok = ld_acquire(&P.draws[(size_t)u.b * (K + 1) + n]);
+            m = __ldcg(&P.draw_mass[(size_t)u.b * (K + 1) + n]);
+        }
+        P.n_acc[u.b] = bad ? -1 : n;
+        P.next[u.b] = tok;
+        if (P.rmass) P.rmass[u.b] = bad ? 0.f : (n == u.L ? 1.f : m);
+        P.arrive[u.b] = 0;                      // ready for the next call
+    }
+    // positions the method never looks at report zeros
+    if (P.ratio)
+        for (int j = u.L + lane; j < K; j += 32) P.ratio[(size_t)u.b * K + j] = 0.f;
+    if (P.stats)
+        for (int j = (u.L + 1) * 4 + lane; j < (K + 1) * 4; j += 32) P.stats[(size_t)u.b * (K + 1) * 4 + j] = 0.f;
+}
+
+}  // namespace sd

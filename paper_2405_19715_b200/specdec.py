@@ -1,0 +1,202 @@
+"""Thin ctypes binding of libspecdec: argument marshalling only, every step runs in the CUDA
+library.  Function names match the C ABI in include/specdec.h.  Tensors are torch CUDA
+tensors (torch is used for device memory and streams only); the *_host variant takes pinned
+CPU tensors.  There is no CPU fallback: a missing library or device raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import torch
+
+from . import build as _build
+
+F32, BF16 = 0, 1
+OK, EINVAL, EUNSUPPORTED, ECUDA, EDATA = 0, 1, 2, 3, 4
+VERIFY_AUTO, VERIFY_DIRECT, VERIFY_STREAM = 0, 1, 2
+DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT = 1, 2, 4
+
+EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
+           "specdec_launch_count", "specdec_verify_correct", "specdec_verify_correct_host",
+           "specdec_accept_head", "specdec_stop"]
+
+
+class SpecdecError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"specdec error {code}: {msg}")
+        self.code = code
+
+
+class _Head(C.Structure):
+    _fields_ = [("W", C.POINTER(C.c_void_p)), ("b", C.POINTER(C.c_void_p)), ("w_out", C.c_void_p),
+                ("b_out", C.c_float), ("d", C.c_int), ("depth", C.c_int)]
+
+
+_lib = None
+
+
+def load_library(path: str | Path | None = None) -> C.CDLL:
+    """Load (building first if the sources are newer) libspecdec.so; raises if that fails."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = Path(path) if path else _build.build()
+    lib = C.CDLL(str(p))
+    vp, ip, fp = C.c_void_p, C.c_void_p, C.c_void_p
+    lib.specdec_create.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int, C.c_int, C.c_int]
+    lib.specdec_destroy.argtypes = [C.c_void_p]
+    lib.specdec_last_error.argtypes = [C.c_void_p]
+    lib.specdec_last_error.restype = C.c_char_p
+    lib.specdec_device_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint32)]
+    lib.specdec_launch_count.argtypes = [C.c_void_p]
+    lib.specdec_launch_count.restype = C.c_uint64
+    lib.specdec_verify_correct.argtypes = [C.c_void_p, vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int, C.c_int,
+                                           C.c_int, ip, ip, fp, fp, fp, C.c_uint32, C.c_void_p]
+    lib.specdec_verify_correct_host.argtypes = [C.c_void_p, vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int,
+                                                C.c_int, C.c_int, ip, ip, fp, C.c_uint32, C.c_void_p]
+    lib.specdec_accept_head.argtypes = [C.c_void_p, vp, C.POINTER(_Head), C.c_int, C.c_int, fp, C.c_void_p]
+    lib.specdec_stop.argtypes = [C.c_void_p, fp, ip, C.c_float, C.c_int, C.c_int, ip, C.c_void_p]
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _ptr(t: torch.Tensor | None, dtype=None, cuda=True) -> int | None:
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected {dtype}, got {t.dtype}")
+    if cuda != t.is_cuda:
+        raise ValueError("tensor is on the wrong side (device vs host)")
+    return t.data_ptr()
+
+
+def _logit_dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise ValueError(f"logits must be float32 or bfloat16, got {t.dtype}")
+
+
+def _stream(stream) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+class Context:
+    """Owns a specdec_ctx.  One context serves one stream at a time."""
+
+    def __init__(self, max_B: int, max_K: int, max_d: int = 0, device: int | None = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libspecdec needs a CUDA device; there is no CPU path")
+        self.lib = load_library()
+        self.device = torch.cuda.current_device() if device is None else device
+        h = C.c_void_p()
+        rc = self.lib.specdec_create(C.byref(h), self.device, max_B, max_K, max_d)
+        if rc != OK:
+            raise SpecdecError(rc, "specdec_create failed")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            self.lib.specdec_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int):
+        if rc != OK:
+            raise SpecdecError(rc, self.lib.specdec_last_error(self.handle).decode())
+
+    def launch_count(self) -> int:
+        return int(self.lib.specdec_launch_count(self.handle))
+
+    def device_status(self, stream=None) -> int:
+        """Synchronises the stream; returns the SPECDEC_DATA_* bits (0 = clean) and clears them."""
+        bits = C.c_uint32(0)
+        rc = self.lib.specdec_device_status(self.handle, _stream(stream), C.byref(bits))
+        if rc not in (OK, EDATA):
+            self._check(rc)
+        return int(bits.value)
+
+
+def specdec_verify_correct(ctx: Context, target_logits, draft_logits, cand_tokens, cand_len, uniforms,
+                           temperature: float, n_accepted=None, next_token=None, accept_ratio=None,
+                           row_stats=None, resid_mass=None, flags: int = VERIFY_AUTO, stream=None):
+    """specdec_verify_correct of the C ABI.  Returns (n_accepted, next_token) device tensors
+    (allocated here unless passed in)."""
+    B, K1, V = target_logits.shape
+    K = K1 - 1
+    if tuple(draft_logits.shape) != (B, K, V) or draft_logits.dtype != target_logits.dtype:
+        raise ValueError("draft_logits must be [B, K, V] of the target's dtype")
+    dev = target_logits.device
+    if n_accepted is None:
+        n_accepted = torch.empty(B, dtype=torch.int32, device=dev)
+    if next_token is None:
+        next_token = torch.empty(B, dtype=torch.int32, device=dev)
+    rc = ctx.lib.specdec_verify_correct(
+        ctx.handle, _ptr(target_logits), _ptr(draft_logits), _logit_dtype(target_logits),
+        _ptr(cand_tokens, torch.int32), _ptr(cand_len, torch.int32), _ptr(uniforms, torch.float32),
+        float(temperature), B, K, V, _ptr(n_accepted, torch.int32), _ptr(next_token, torch.int32),
+        _ptr(accept_ratio, torch.float32), _ptr(row_stats, torch.float32), _ptr(resid_mass, torch.float32),
+        flags, _stream(stream))
+    ctx._check(rc)
+    return n_accepted, next_token
+
+
+def specdec_verify_correct_host(ctx: Context, target_logits, draft_logits, cand_tokens, cand_len, uniforms,
+                                temperature: float, n_accepted=None, next_token=None, accept_ratio=None,
+                                flags: int = VERIFY_AUTO, stream=None):
+    """specdec_verify_correct_host of the C ABI: all tensors live in (pinned) host memory; returns
+    host tensors after the stream has been synchronised."""
+    B, K1, V = target_logits.shape
+    K = K1 - 1
+    if n_accepted is None:
+        n_accepted = torch.empty(B, dtype=torch.int32).pin_memory()
+    if next_token is None:
+        next_token = torch.empty(B, dtype=torch.int32).pin_memory()
+    rc = ctx.lib.specdec_verify_correct_host(
+        ctx.handle, _ptr(target_logits, cuda=False), _ptr(draft_logits, cuda=False), _logit_dtype(target_logits),
+        _ptr(cand_tokens, torch.int32, False), _ptr(cand_len, torch.int32, False),
+        _ptr(uniforms, torch.float32, False), float(temperature), B, K, V,
+        _ptr(n_accepted, torch.int32, False), _ptr(next_token, torch.int32, False),
+        _ptr(accept_ratio, torch.float32, False), flags, _stream(stream))
+    ctx._check(rc)
+    return n_accepted, next_token
+
+
+def specdec_accept_head(ctx: Context, hidden, W, b, w_out, b_out: float, accept_prob=None, stream=None):
+    """specdec_accept_head of the C ABI.  hidden [B,K,d] bf16; W: list of [d,d] bf16; b: list of
+    [d] bf16 or None entries (or None); w_out [d] bf16.  Returns accept_prob [B,K] fp32."""
+    B, K, d = hidden.shape
+    depth = len(W)
+    Wp = (C.c_void_p * max(depth, 1))(*[_ptr(w, torch.bfloat16) for w in W])
+    bl = list(b) if b is not None else [None] * depth
+    bp = (C.c_void_p * max(depth, 1))(*[_ptr(x, torch.bfloat16) for x in bl])
+    head = _Head(C.cast(Wp, C.POINTER(C.c_void_p)), C.cast(bp, C.POINTER(C.c_void_p)),
+                 _ptr(w_out, torch.bfloat16), float(b_out), d, depth)
+    if accept_prob is None:
+        accept_prob = torch.empty(B, K, dtype=torch.float32, device=hidden.device)
+    rc = ctx.lib.specdec_accept_head(ctx.handle, _ptr(hidden, torch.bfloat16), C.byref(head), B, K,
+                                     _ptr(accept_prob, torch.float32), _stream(stream))
+    ctx._check(rc)
+    return accept_prob
+
+
+def specdec_stop(ctx: Context, accept_prob, h: float, cand_len=None, stop_pos=None, stream=None):
+    """specdec_stop of the C ABI.  Returns stop_pos [B] int32."""
+    B, K = accept_prob.shape
+    if stop_pos is None:
+        stop_pos = torch.empty(B, dtype=torch.int32, device=accept_prob.device)
+    rc = ctx.lib.specdec_stop(ctx.handle, _ptr(accept_prob, torch.float32), _ptr(cand_len, torch.int32),
+                              float(h), B, K, _ptr(stop_pos, torch.int32), _stream(stream))
+    ctx._check(rc)
+    return stop_pos

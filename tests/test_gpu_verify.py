@@ -1,0 +1,236 @@
+"""GPU parity of specdec_verify_correct / specdec_stop against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from paper_2405_19715_b200 import specdec, workloads as wl  # noqa: E402
+from tests import parity  # noqa: E402
+
+KERNELS = [specdec.VERIFY_DIRECT, specdec.VERIFY_STREAM]
+KERNEL_IDS = ["direct", "stream"]
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = specdec.Context(max_B=256, max_K=32)
+    yield c
+    c.close()
+
+
+def _stream_ok(inp):
+    V = inp["target_logits"].shape[-1]
+    es = 2 if inp["target_logits"].dtype == np.uint16 else 4
+    return (V * es) % 16 == 0
+
+
+def _random_problem(seed, B, K, V, dtype, T=1.0, sigma_n=1.0, ragged=True):
+    cfg = wl.Workload(f"t{seed}", B=B, K=K, V=V, dtype=dtype, sigma_d=2.5, sigma_n=sigma_n, T=T, ragged=ragged, seed=seed)
+    inp = wl.make_verify_inputs(cfg, threads=1)
+    if ragged and B >= 3:        # make sure the degenerate lengths appear
+        lens = inp["cand_len"].copy()
+        lens[0], lens[1] = 0, K
+        cfg2 = cfg
+        inp = wl.make_verify_inputs(cfg2, threads=1)
+        # re-poison consistently for the changed lengths by regenerating row by row
+        for b in (0, 1):
+            t, d, y = wl._row_logits(cfg, b, int(lens[b]), cfg.sigma_n, False)
+            inp["target_logits"][b], inp["draft_logits"][b], inp["cand_tokens"][b] = t, d, y
+        inp["cand_len"] = lens
+    return inp
+
+
+@pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [1, 2, 7, 8, 33, 1000, 4104, 20000])
+@pytest.mark.parametrize("K", [1, 2, 16])
+def test_small_shapes(ctx, V, K, dtype, flags):
+    inp = _random_problem(1000 + V + K, B=5, K=K, V=V, dtype=dtype, T=0.9)
+    if flags == specdec.VERIFY_STREAM and not _stream_ok(inp):
+        pytest.skip("rows not 16-byte aligned: served by the direct kernel")
+    gpu = parity.run_gpu_verify(ctx, inp, flags)
+    rep = parity.classify_rows(inp, gpu, dtype="f32")      # bf16 inputs are widened exactly: same bar
+    assert ctx.device_status() == 0
+    assert rep["exact"] + rep["boundary_n"] + rep["boundary_token"] == 5
+
+
+@pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
+@pytest.mark.parametrize("name", ["cfg1", "cfg2", "cfg3"])
+def test_configs_1_to_3(ctx, name, flags):
+    cfg = wl.CONFIGS[name]
+    inp = wl.make_verify_inputs(cfg)
+    gpu = parity.run_gpu_verify(ctx, inp, flags)
+    rep = parity.classify_rows(inp, gpu, dtype="f32")
+    print(name, rep)
+    assert ctx.device_status() == 0
+    # the same call again must give bit-identical outputs (no order-dependent race)
+    gpu2 = parity.run_gpu_verify(ctx, inp, flags)
+    for k in ("n_accepted", "next_token", "accept_ratio", "row_stats", "resid_mass"):
+        assert np.array_equal(gpu[k], gpu2[k]), k
+
+
+@pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
+def test_config4_full_size_sampled_rows(ctx, flags):
+    """Full-size cfg4 (B=256, K=16, V=128256, bf16) in the launch configuration the benchmark times;
+    the oracle checks a sample of rows (peaked and ordinary) one by one, properties cover the rest."""
+    cfg = wl.CONFIGS["cfg4"]
+    inp = wl.make_verify_inputs(cfg)
+    gpu = parity.run_gpu_verify(ctx, inp, flags)
+    assert ctx.device_status() == 0
+    peaked = np.nonzero(inp["peaked"])[0]
+    plain = np.nonzero(~inp["peaked"])[0]
+    rows = list(peaked[:3]) + list(plain[:5]) + [int(plain[-1])]
+    rep = parity.classify_rows(inp, gpu, rows=rows, dtype="f32")
+    print("cfg4", rep)
+    n, tok = gpu["n_accepted"], gpu["next_token"]
+    assert np.all((n >= 0) & (n <= cfg.K)) and np.all((tok >= 0) & (tok < cfg.V))
+    # rows whose drafted tokens carry +12 on the target are accepted almost surely
+    assert (n[peaked] == cfg.K).mean() > 0.8
+    # accept ratios decide n: first position with r >= ratio
+    r = inp["uniforms"][:, :cfg.K]
+    rej = r >= gpu["accept_ratio"]
+    first = np.where(rej.any(1), rej.argmax(1), cfg.K)
+    assert np.array_equal(first, n)
+    # the drawn token has positive residual weight: p(y') > q(y') needs the logits only up to lse,
+    # checked on the sampled rows by the oracle; here every row's mass is within (0, 1]
+    assert np.all((gpu["resid_mass"] > 0) & (gpu["resid_mass"] <= 1.0 + 1e-5))
+
+
+@pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
+def test_special_cases(ctx, flags):
+    rng = np.random.default_rng(3)
+    B, K, V = 6, 5, 4096
+    d = rng.normal(scale=3, size=(B, K, V)).astype(np.float32)
+    t = np.concatenate([d, rng.normal(size=(B, 1, V)).astype(np.float32)], axis=1)
+    y = rng.integers(0, V, size=(B, K)).astype(np.int32)
+    u = wl.uniforms_24bit(rng, (B, K + 1))
+    base = dict(target_logits=t, draft_logits=d, cand_tokens=y, cand_len=None, uniforms=u, temperature=np.float32(1.0))
+    # identical models: everything accepted, bonus draw from p_{K+1}
+    gpu = parity.run_gpu_verify(ctx, base, flags)
+    assert np.all(gpu["n_accepted"] == K) and np.all(gpu["accept_ratio"] == 1.0)
+    parity.classify_rows(base, gpu, dtype="f32")
+    # very high temperature: both uniform
+    hot = dict(base, target_logits=rng.normal(size=(B, K + 1, V)).astype(np.float32), temperature=np.float32(1e30))
+    assert np.all(parity.run_gpu_verify(ctx, hot, flags)["n_accepted"] == K)
+    # target one-hot on a token the draft did not pick: certain rejection, residual is a point mass
+    t3 = t.copy()
+    other = (y + 1) % V
+    for b in range(B):
+        t3[b, np.arange(K), other[b]] += 200.0
+    peaked = dict(base, target_logits=t3)
+    gpu = parity.run_gpu_verify(ctx, peaked, flags)
+    assert np.all(gpu["n_accepted"] == 0) and np.array_equal(gpu["next_token"], other[:, 0])
+    parity.classify_rows(peaked, gpu, dtype="f32")
+    # masked (-inf) logits and huge offsets do not break the statistics
+    t4, d4 = t.copy(), d.copy()
+    t4[:, :, :100] = -np.inf
+    d4[:, :, :100] = -np.inf
+    t4[:, :, 100:] += 3.0e4
+    y4 = np.maximum(y, 100).astype(np.int32)
+    masked = dict(base, target_logits=t4, draft_logits=d4, cand_tokens=y4)
+    gpu = parity.run_gpu_verify(ctx, masked, flags)
+    parity.classify_rows(masked, gpu, dtype="f32")
+    assert np.all(gpu["next_token"] >= 100)
+    # low temperature approaches greedy decoding
+    cold = dict(base, target_logits=t + rng.normal(scale=1.0, size=t.shape).astype(np.float32),
+                cand_tokens=d.argmax(-1).astype(np.int32), temperature=np.float32(0.05))
+    gpu = parity.run_gpu_verify(ctx, cold, flags)
+    parity.classify_rows(cold, gpu, dtype="f32")
+
+
+@pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
+def test_outputs_ignore_positions_after_first_rejection(ctx, flags):
+    cfg = wl.Workload("inv", B=16, K=8, V=8192, dtype="bf16", sigma_d=3.0, sigma_n=1.5, T=1.0, seed=77)
+    inp = wl.make_verify_inputs(cfg)
+    g1 = parity.run_gpu_verify(ctx, inp, flags)
+    inp2 = {k: (v.copy() if isinstance(v, np.ndarray) else v) for k, v in inp.items()}
+    rng = np.random.default_rng(1)
+    for b in range(cfg.B):
+        n = g1["n_accepted"][b]
+        inp2["target_logits"][b, n + 1:] = wl.f32_to_bf16_bits(rng.normal(scale=9, size=inp2["target_logits"][b, n + 1:].shape).astype(np.float32))
+        inp2["draft_logits"][b, n + 1:] = wl.f32_to_bf16_bits(rng.normal(scale=9, size=inp2["draft_logits"][b, n + 1:].shape).astype(np.float32))
+        inp2["cand_tokens"][b, n + 1:] = (inp2["cand_tokens"][b, n + 1:] + 1) % cfg.V
+    g2 = parity.run_gpu_verify(ctx, inp2, flags)
+    assert np.array_equal(g1["n_accepted"], g2["n_accepted"]) and np.array_equal(g1["next_token"], g2["next_token"])
+
+
+@pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
+def test_bad_data_sets_status_without_trapping(ctx, flags):
+    cfg = wl.Workload("bad", B=6, K=4, V=2048, dtype="bf16", sigma_d=3.0, sigma_n=1.0, T=1.0, seed=5)
+    inp = wl.make_verify_inputs(cfg)
+    inp["cand_len"] = np.array([4, 9, 4, -1, 4, 4], np.int32)
+    inp["cand_tokens"][2, 1] = cfg.V
+    inp["cand_tokens"][4, 0] = -3
+    gpu = parity.run_gpu_verify(ctx, inp, flags)
+    assert ctx.device_status() == (specdec.DATA_BAD_LENGTH | specdec.DATA_BAD_TOKEN)
+    assert ctx.device_status() == 0                       # reading clears it
+    for b in (1, 2, 3, 4):
+        assert gpu["n_accepted"][b] == -1 and gpu["next_token"][b] == -1
+    good = dict(inp, cand_len=np.array([4, 4, 4, 4, 4, 4], np.int32))
+    rep = parity.classify_rows(good, gpu, rows=[0, 5], dtype="f32")
+    assert rep["rows"] == 2
+    # the context still works afterwards
+    inp_ok = wl.make_verify_inputs(cfg)
+    parity.classify_rows(inp_ok, parity.run_gpu_verify(ctx, inp_ok, flags), dtype="f32")
+
+
+def test_argument_errors(ctx):
+    t = torch.zeros(2, 3, 64, device="cuda")
+    d = torch.zeros(2, 2, 64, device="cuda")
+    y = torch.zeros(2, 2, dtype=torch.int32, device="cuda")
+    u = torch.zeros(2, 3, device="cuda")
+    with pytest.raises(specdec.SpecdecError) as e:
+        specdec.specdec_verify_correct(ctx, t, d, y, None, u, 0.0)
+    assert e.value.code == specdec.EINVAL
+    with pytest.raises(specdec.SpecdecError) as e:
+        specdec.specdec_verify_correct(ctx, t, d, y, None, u, float("nan"))
+    assert e.value.code == specdec.EINVAL
+    big = torch.zeros(300, 3, 8, device="cuda")
+    with pytest.raises(specdec.SpecdecError) as e:
+        specdec.specdec_verify_correct(ctx, big, torch.zeros(300, 2, 8, device="cuda"),
+                                       torch.zeros(300, 2, dtype=torch.int32, device="cuda"), None,
+                                       torch.zeros(300, 3, device="cuda"), 1.0)
+    assert e.value.code == specdec.EUNSUPPORTED
+    with pytest.raises(specdec.SpecdecError) as e:   # 66 bf16 = 132 bytes per row: not 16-byte aligned
+        specdec.specdec_verify_correct(ctx, torch.zeros(2, 3, 66, device="cuda", dtype=torch.bfloat16),
+                                       torch.zeros(2, 2, 66, device="cuda", dtype=torch.bfloat16), y, None, u, 1.0,
+                                       flags=specdec.VERIFY_STREAM)
+    assert e.value.code == specdec.EUNSUPPORTED
+
+
+def test_host_entry_point_matches_device_entry_point(ctx):
+    cfg = wl.CONFIGS["cfg2"]
+    inp = wl.make_verify_inputs(cfg)
+    gpu = parity.run_gpu_verify(ctx, inp)
+    h = {k: parity.to_torch(np.ascontiguousarray(inp[k]), "cpu", pin=True)
+         for k in ("target_logits", "draft_logits", "cand_tokens", "cand_len", "uniforms")}
+    ratio = torch.empty(cfg.B, cfg.K).pin_memory()
+    n, tok = specdec.specdec_verify_correct_host(ctx, h["target_logits"], h["draft_logits"], h["cand_tokens"],
+                                                 h["cand_len"], h["uniforms"], float(inp["temperature"]),
+                                                 accept_ratio=ratio)
+    assert np.array_equal(n.numpy(), gpu["n_accepted"]) and np.array_equal(tok.numpy(), gpu["next_token"])
+    assert np.array_equal(ratio.numpy(), gpu["accept_ratio"])
+
+
+def test_stop_rule_parity(ctx):
+    for name, hs in (("cfg1", [0.5]), ("cfg3", [0.3, 0.5, 0.7])):
+        cfg = wl.CONFIGS[name]
+        a = wl.make_accept_prob(cfg)
+        lens = wl.make_cand_len(cfg) if cfg.ragged else None
+        ta = torch.from_numpy(a).cuda()
+        tl = None if lens is None else torch.from_numpy(lens).cuda()
+        for h in hs:
+            pos = specdec.specdec_stop(ctx, ta, h, tl).cpu().numpy()
+            rep = parity.classify_stop(a, h, pos, lens)
+            assert rep["exact"] + rep["boundary"] == cfg.B
+    # thresholds outside (0,1) and rows of ones
+    a = np.ones((4, 7), np.float32)
+    assert np.all(specdec.specdec_stop(ctx, torch.from_numpy(a).cuda(), 0.0).cpu().numpy() == 7)
+    b = np.full((4, 7), 0.9, np.float32)
+    assert np.all(specdec.specdec_stop(ctx, torch.from_numpy(b).cuda(), -0.5).cpu().numpy() == 0)
+    assert np.all(specdec.specdec_stop(ctx, torch.from_numpy(b).cuda(), 1.0).cpu().numpy() == 7)
+    big = np.random.default_rng(0).uniform(0.3, 1.0, size=(3000, 20)).astype(np.float32)
+    pos = specdec.specdec_stop(specdec.Context(3000, 20), torch.from_numpy(big).cuda(), 0.6).cpu().numpy()
+    rep = parity.classify_stop(big, 0.6, pos)
+    assert rep["exact"] + rep["boundary"] == 3000
