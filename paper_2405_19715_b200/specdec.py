@@ -87,6 +87,16 @@ def _stream(stream) -> int:
     return s.cuda_stream
 
 
+def from_numpy(a, device="cuda", pin: bool = False) -> torch.Tensor:
+    """numpy array -> torch tensor (uint16 arrays are bfloat16 bit patterns); marshalling only."""
+    import numpy as np
+    a = np.ascontiguousarray(a)
+    t = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)
+    if str(device) == "cpu":
+        return t.pin_memory() if pin else t
+    return t.to(device)
+
+
 class Context:
     """Owns a specdec_ctx.  One context serves one stream at a time."""
 

@@ -97,7 +97,7 @@ def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
 
 
 def _store(x: np.ndarray, dtype: str) -> np.ndarray:
-    return f32_to_bf16_bits(x) if dtype == "bf16" else np.ascontiguousarray(x, dtype=np.float32)
+    return f32_to_bf16_bits(x) if dtype == "bf16" else np.array(x, dtype=np.float32, order="C", copy=True)
 
 
 def _stored_as_f32(x: np.ndarray, dtype: str) -> np.ndarray:

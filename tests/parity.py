@@ -17,14 +17,7 @@ BOUNDARY = 1e-6
 PROB_RTOL = {"f32": 1e-5, "bf16": 2e-2}     # spec tolerances on probabilities
 
 
-def to_torch(a: np.ndarray, device="cuda", pin=False):
-    if a.dtype == np.uint16:
-        t = torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
-    else:
-        t = torch.from_numpy(a)
-    if device == "cpu":
-        return t.pin_memory() if pin else t
-    return t.to(device)
+to_torch = specdec.from_numpy
 
 
 def run_gpu_verify(ctx, inp, flags=0, want_stats=True):
@@ -118,9 +111,11 @@ def classify_rows(inp, gpu, rows=None, dtype="bf16", check_probs=True):
                 gm, om = gpu["resid_mass"][b], o["resid_mass"][k]
                 rel = abs(gm - om) / max(om, 1e-30)
                 rep["max_mass_rel"] = max(rep["max_mass_rel"], rel)
-                assert rel <= max(rtol, 1e-5), f"row {b}: residual mass {gm!r} vs {om!r}"
+                # W = sum (p-q)_+ cancels: fp32 probabilities carry ~1e-7 each, so the bound is absolute
+                assert abs(gm - om) <= rtol * om + 1e-6, f"row {b}: residual mass {gm!r} vs {om!r}"
                 if gn == L:
-                    assert abs(st[L, 0] - o["lse_p"][k, L]) <= 1e-5 * max(1.0, abs(o["lse_p"][k, L]))
+                    assert abs(st[L, 0] - o["lse_p"][k, L]) <= 1e-5 * max(1.0, abs(o["lse_p"][k, L])), \
+                        f"row {b}: bonus lse {st[L, 0]!r} vs {o['lse_p'][k, L]!r} (L={L}, stats={st.tolist()})"
     return rep
 
 
