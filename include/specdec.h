@@ -28,6 +28,7 @@
 #ifndef SPECDEC_H_
 #define SPECDEC_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -168,6 +169,39 @@ int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const specdec_head
  */
 int specdec_stop(specdec_ctx* ctx, const float* accept_prob, const int32_t* cand_len,
                  float h, int B, int K, int32_t* stop_pos, void* stream);
+
+/*
+ * Allocation-free variant of specdec_verify_correct.  The paper has no counterpart: this entry
+ * point exists for callers that cannot call cudaMalloc -- a serving process that has given all
+ * device memory to its own pool, a plugin whose host forbids allocations after start-up, a
+ * latency-critical loop that cannot afford an allocation's implicit synchronisation.  It needs
+ * no context (creating one allocates).  Its scratch is one fixed array of about 256 KB inside
+ * the library's device image, present on every GPU that loads the library until the process ends.
+ *
+ * Inputs and outputs are as for specdec_verify_correct (all "dev", on the CURRENT device),
+ * without the optional probability outputs.  data_status (dev, may be NULL) is a word the caller
+ * has zeroed; SPECDEC_DATA_* bits are OR-ed into it when a token or length is out of range.
+ * err/err_len: host buffer that receives a message when the return value is not SPECDEC_OK
+ * (may be NULL/0).
+ *
+ * Limits: B * (K+1) <= SPECDEC_STATIC_MAX_UNITS and V <= SPECDEC_STATIC_MAX_V; larger problems
+ * return SPECDEC_EUNSUPPORTED with a message and launch nothing.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, no
+ * allocation); make that first call outside any stream capture.  Every call on a device shares
+ * the one array, which keeps the previous call's contents: the library clears what must start
+ * from zero on `stream` before the kernel, so calls on one stream are safe back to back, but two
+ * calls whose GPU work overlaps (different streams, different host threads) race on it and give
+ * wrong results.  Calls no cudaMalloc, cudaFree or any other allocating routine.
+ */
+#define SPECDEC_STATIC_MAX_UNITS 16384
+#define SPECDEC_STATIC_MAX_V     262144
+int specdec_verify_correct_static(const void* target_logits, const void* draft_logits, specdec_dtype dtype,
+                                  const int32_t* cand_tokens, const int32_t* cand_len,
+                                  const float* uniforms, float temperature,
+                                  int B, int K, int V,
+                                  int32_t* n_accepted, int32_t* next_token,
+                                  uint32_t* data_status, void* stream, char* err, size_t err_len);
 
 #ifdef __cplusplus
 }

@@ -19,7 +19,8 @@ DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT = 1, 2, 4
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
            "specdec_launch_count", "specdec_verify_correct", "specdec_verify_correct_host",
-           "specdec_accept_head", "specdec_stop"]
+           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static"]
+STATIC_MAX_UNITS, STATIC_MAX_V = 16384, 262144
 
 
 class SpecdecError(RuntimeError):
@@ -57,6 +58,8 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
                                                 C.c_int, C.c_int, ip, ip, fp, C.c_uint32, C.c_void_p]
     lib.specdec_accept_head.argtypes = [C.c_void_p, vp, C.POINTER(_Head), C.c_int, C.c_int, fp, C.c_void_p]
     lib.specdec_stop.argtypes = [C.c_void_p, fp, ip, C.c_float, C.c_int, C.c_int, ip, C.c_void_p]
+    lib.specdec_verify_correct_static.argtypes = [vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int, C.c_int, C.c_int,
+                                                  ip, ip, C.c_void_p, C.c_void_p, C.c_char_p, C.c_size_t]
     if path is None:
         _lib = lib
     return lib
@@ -210,3 +213,22 @@ def specdec_stop(ctx: Context, accept_prob, h: float, cand_len=None, stop_pos=No
                               float(h), B, K, _ptr(stop_pos, torch.int32), _stream(stream))
     ctx._check(rc)
     return stop_pos
+
+
+def specdec_verify_correct_static(target_logits, draft_logits, cand_tokens, cand_len, uniforms, temperature: float,
+                                  n_accepted, next_token, data_status=None, stream=None):
+    """specdec_verify_correct_static of the C ABI: verify/correct without a context and without any
+    allocation inside the library, for callers that may not call cudaMalloc (every device buffer,
+    outputs included, is passed in).  B*(K+1) <= STATIC_MAX_UNITS and V <= STATIC_MAX_V; calls
+    whose GPU work overlaps share one scratch array and race."""
+    lib = load_library()
+    B, K1, V = target_logits.shape
+    err = C.create_string_buffer(256)
+    rc = lib.specdec_verify_correct_static(
+        _ptr(target_logits), _ptr(draft_logits), _logit_dtype(target_logits), _ptr(cand_tokens, torch.int32),
+        _ptr(cand_len, torch.int32), _ptr(uniforms, torch.float32), float(temperature), B, K1 - 1, V,
+        _ptr(n_accepted, torch.int32), _ptr(next_token, torch.int32),
+        None if data_status is None else data_status.data_ptr(), _stream(stream), err, len(err))
+    if rc != OK:
+        raise SpecdecError(rc, err.value.decode())
+    return n_accepted, next_token
