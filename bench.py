@@ -270,15 +270,19 @@ def run_ours(args, cfg):
         specdec.specdec_verify_correct_host(ctx, host["target_logits"], host["draft_logits"], host["cand_tokens"],
                                             host["cand_len"], host["uniforms"], T, h_n, h_t, flags=args.kernel)
 
-    e2e_step()
-    torch.cuda.synchronize()
-    barrier(world)
-    e0.record()
-    for _ in range(e2e_steps):
+    if args.no_e2e:
+        e2e_steps = 0
+        e2e_ms = float("nan")
+    else:
         e2e_step()
-    e1.record()
-    torch.cuda.synchronize()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / e2e_steps
+        torch.cuda.synchronize()
+        barrier(world)
+        e0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        e1.record()
+        torch.cuda.synchronize()
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / e2e_steps
     h2d = sum(v.numel() * v.element_size() for v in host.values()) + h_acc.numel() * 4 + host["cand_len"].numel() * 4
     d2h = 3 * cfg.B * 4
 
@@ -319,8 +323,12 @@ def main():
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 direct, 2 stream")
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling runs)")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.workload]
+    if args.batch:
+        cfg = cfg.scaled(B=args.batch, name=f"{cfg.name}(B={args.batch})")
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

@@ -69,6 +69,10 @@ int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_
     if (e == cudaSuccess) e = cudaMalloc(&ctx->draw_mass, ndraw * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->arrive, (size_t)max_B * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->status, sizeof(uint32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->norms, ndraw * sizeof(float4));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->tasks, (size_t)max_B * sizeof(int2));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->task_ctl, 2 * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->task_ctl, 0, 2 * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->flags, 0, nflag * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->arrive, 0, (size_t)max_B * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
@@ -96,6 +100,9 @@ int specdec_destroy(specdec_ctx* ctx) {
     cudaFree(ctx->draw_mass);
     cudaFree(ctx->arrive);
     cudaFree(ctx->status);
+    cudaFree(ctx->norms);
+    cudaFree(ctx->tasks);
+    cudaFree(ctx->task_ctl);
     cudaFree(ctx->stage);
     cudaFree(ctx->act[0]);
     cudaFree(ctx->act[1]);
@@ -156,6 +163,9 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
     p.draw_mass = ctx->draw_mass;
     p.arrive = ctx->arrive;
     p.status = ctx->status;
+    p.norms = ctx->norms;
+    p.tasks = ctx->tasks;
+    p.task_ctl = ctx->task_ctl;
     p.epoch = ctx->epoch;
 
     const bool stream_ok = verify_stream_supported(p, dtype);

@@ -16,6 +16,9 @@ struct specdec_ctx {
     float* draw_mass = nullptr;   // [max_B * (max_K+1)]  mass of the weights that draw came from
     int32_t* arrive = nullptr;    // [max_B]              positions of a row that have finished
     uint32_t* status = nullptr;   // sticky SPECDEC_DATA_* bits
+    float4* norms = nullptr;      // [max_B * (max_K+1)]  log2 normalisers {hi_p, lo_p, hi_q, lo_q} per position
+    int2* tasks = nullptr;        // [max_B]              rows whose y' is still to be drawn: {b, n}
+    int32_t* task_ctl = nullptr;  // [2]                  {number of tasks, CTAs of the draw kernel that finished}
     uint32_t epoch = 0;
     uint64_t launches = 0;
     // staging for the host-buffer entry point (device), grown on demand
@@ -45,6 +48,9 @@ struct VerifyParams {
     float* draw_mass;
     int32_t* arrive;
     uint32_t* status;
+    float4* norms;
+    int2* tasks;
+    int32_t* task_ctl;
     uint32_t epoch;
 };
 

@@ -83,17 +83,19 @@ __global__ void __launch_bounds__(DIRECT_THREADS, 2) verify_direct_kernel(const 
         Acc a = lane < NW ? sh.wp[lane] : acc_init(), b = lane < NW ? sh.wq[lane] : acc_init();
         a = warp_merge(a);
         b = warp_merge(b);
+        int y = 0, y_ok = 1;
+        float t_y = 0.f, d_y = 0.f, r = 0.f;
+        if (lane == 0 && !u.bonus) {
+            r = P.uniforms[(size_t)u.b * (P.K + 1) + u.i];
+            y = P.tokens[(size_t)u.b * P.K + u.i];
+            y_ok = (y >= 0 && y < P.V);
+            if (y_ok) { t_y = to_float(trow[y]); d_y = to_float(drow[y]); }
+        }
+        const int mode = unit_decide(P, u, a, b, t_y, d_y, y_ok, r, lane);
         if (lane == 0) {
-            int y = 0, y_ok = 1;
-            float t_y = 0.f, d_y = 0.f;
-            if (!u.bonus) {
-                y = P.tokens[(size_t)u.b * P.K + u.i];
-                y_ok = (y >= 0 && y < P.V);
-                if (y_ok) { t_y = to_float(trow[y]); d_y = to_float(drow[y]); }
-            }
             sh.np = make_norm(a);
             sh.nq = u.bonus ? sh.np : make_norm(b);
-            sh.need_draw = unit_decide(P, u, a, b, t_y, d_y, y_ok);
+            sh.need_draw = mode;
         }
     }
     __syncthreads();

@@ -33,6 +33,19 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
 __device__ __forceinline__ void st_release(int32_t* p, int v) {
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+__device__ __forceinline__ int ld_relaxed(const int32_t* p) {
+    int v;
+    asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_relaxed(int32_t* p, int v) {
+    asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int atom_add_acq_rel(int32_t* p, int v) {
+    int old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
 __device__ __forceinline__ void bar_sync(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
@@ -155,46 +168,60 @@ struct Unit {
     bool bonus;                // i == L: the p_{L+1} row, no draft
 };
 
-// Called by one thread once the unit's statistics are known: accept test, optional outputs,
-// flag publication and the decision whether this unit must produce a draw.
-__device__ __forceinline__ int unit_decide(const VerifyParams& P, const Unit& u, const Acc& ap, const Acc& aq,
-                                           float t_y, float d_y, int y_ok) {
+// Accept test of one unit, called by one full warp once the unit's statistics are known (they
+// only need to be valid in lane 0, as do t_y, d_y, y_ok and r = uniforms[b, i]): optional
+// outputs and flag publication.  Returns the flag state (0 for the bonus unit) in every lane.
+// Flags are plain gpu-scope stores: a flag is self-contained (it carries the call's epoch), and
+// the row's arrival counter orders it for the final ballot.
+__device__ __forceinline__ int unit_accept(const VerifyParams& P, const Unit& u, const Acc& ap, const Acc& aq,
+                                           float t_y, float d_y, int y_ok, float r, int lane) {
     const int K = P.K;
     const float LN2 = 0.6931471805599453f;
     int state = 0;
-    if (!u.bonus) {
-        // log2 p(y) and log2 q(y); the references cancel exactly because each term is formed
-        // against the same rs the sum was accumulated with.
-        const float lp = fmaf(t_y, P.c, -ap.rs) - log2f(ap.s);
-        const float lq = fmaf(d_y, P.c, -aq.rs) - log2f(aq.s);
-        const float ratio = exp2f(lp - lq);
-        const float r = P.uniforms[(size_t)u.b * (K + 1) + u.i];
-        state = !y_ok ? FLAG_BAD : (r >= ratio ? FLAG_REJECT : FLAG_ACCEPT);   // r == ratio rejects
-        if (!y_ok) atomicOr(P.status, SPECDEC_DATA_BAD_TOKEN);
-        if (P.ratio) P.ratio[(size_t)u.b * K + u.i] = y_ok ? fminf(1.f, ratio) : -1.f;
-        if (P.stats) {
-            float4 st;
-            st.x = (ap.rs + log2f(ap.s)) * LN2;
-            st.y = (aq.rs + log2f(aq.s)) * LN2;
-            st.z = exp2f(lp);
-            st.w = exp2f(lq);
+    if (lane == 0) {
+        if (!u.bonus) {
+            // log2 p(y) and log2 q(y); the references cancel exactly because each term is formed
+            // against the same rs the sum was accumulated with.
+            const float lp = fmaf(t_y, P.c, -ap.rs) - log2f(ap.s);
+            const float lq = fmaf(d_y, P.c, -aq.rs) - log2f(aq.s);
+            const float ratio = exp2f(lp - lq);
+            state = !y_ok ? FLAG_BAD : (r >= ratio ? FLAG_REJECT : FLAG_ACCEPT);   // r == ratio rejects
+            if (!y_ok) atomicOr(P.status, SPECDEC_DATA_BAD_TOKEN);
+            if (P.ratio) P.ratio[(size_t)u.b * K + u.i] = y_ok ? fminf(1.f, ratio) : -1.f;
+            if (P.stats) {
+                float4 st;
+                st.x = (ap.rs + log2f(ap.s)) * LN2;
+                st.y = (aq.rs + log2f(aq.s)) * LN2;
+                st.z = exp2f(lp);
+                st.w = exp2f(lq);
+                reinterpret_cast<float4*>(P.stats)[(size_t)u.b * (K + 1) + u.i] = st;
+            }
+            st_relaxed(&P.flags[(size_t)u.b * K + u.i], (int)((P.epoch << 2) | (uint32_t)state));
+        } else if (P.stats) {
+            float4 st = make_float4((ap.rs + log2f(ap.s)) * LN2, 0.f, 0.f, 0.f);
             reinterpret_cast<float4*>(P.stats)[(size_t)u.b * (K + 1) + u.i] = st;
         }
-        st_release(&P.flags[(size_t)u.b * K + u.i], (int)((P.epoch << 2) | (uint32_t)state));
-    } else if (P.stats) {
-        float4 st = make_float4((ap.rs + log2f(ap.s)) * LN2, 0.f, 0.f, 0.f);
-        reinterpret_cast<float4*>(P.stats)[(size_t)u.b * (K + 1) + u.i] = st;
     }
-    // A draw is needed only if this position can be the first rejection (or the bonus draw):
-    // skip it when an earlier position of the row is already known to have rejected.
+    return __shfl_sync(0xffffffffu, state, 0);
+}
+
+// Accept test plus the decision whether this unit must produce a draw itself (kernels that draw
+// inside the unit): 0 none, 1 from the residual, 2 from the target (bonus position).  A draw is
+// needed only if this position can be the first rejection (or is the bonus position); it is
+// skipped when an earlier position of the row is already known to have rejected.
+__device__ __forceinline__ int unit_decide(const VerifyParams& P, const Unit& u, const Acc& ap, const Acc& aq,
+                                           float t_y, float d_y, int y_ok, float r, int lane) {
+    const int state = unit_accept(P, u, ap, aq, t_y, d_y, y_ok, r, lane);
+    if (!u.bonus && state != FLAG_REJECT) return 0;      // accepted (or bad token): never draws
     bool known = false;
-    for (int j = 0; j < u.i; ++j) {
-        const int f = ld_acquire(&P.flags[(size_t)u.b * K + j]);
-        if (((uint32_t)f >> 2) == P.epoch && (f & 3) >= FLAG_REJECT) known = true;
+    for (int j0 = 0; j0 < u.i; j0 += 32) {
+        const int j = j0 + lane;
+        int f = 0;
+        if (j < u.i) f = ld_relaxed(&P.flags[(size_t)u.b * P.K + j]);
+        known |= __any_sync(0xffffffffu, ((uint32_t)f >> 2) == P.epoch && (f & 3) >= FLAG_REJECT);
     }
-    if (known || state == FLAG_BAD) return 0;
-    if (u.bonus) return 2;
-    return state == FLAG_REJECT ? 1 : 0;
+    if (known) return 0;
+    return u.bonus ? 2 : 1;
 }
 
 // Weights y' is drawn from, for one vector: (p - q)_+ (mode 1) or p (mode 2).
@@ -209,6 +236,103 @@ __device__ __forceinline__ float vec_weights(const float (&xt)[N], const float (
         sum += w[k];
     }
     return sum;
+}
+
+// Second half of a draw, run by one full warp once every slab sum is in `slab_sum`: fp64 prefix
+// over the slabs, the slab that holds u * total, then a walk inside that slab (its vectors are
+// re-read from global memory).  Returns the token; *total_out receives the total mass.
+template <typename T, bool VEC>
+__device__ __forceinline__ int draw_select(const VerifyParams& P, const T* __restrict__ trow,
+                                           const T* __restrict__ drow, int mode, float u01, const Norm np,
+                                           const Norm nq, const float* __restrict__ slab_sum, int lane,
+                                           double* total_out) {
+    constexpr int N = Elem<T>::EPV;
+    const int V = P.V;
+    const int nvec = (V + N - 1) / N;
+    const int nslab = (nvec + 31) / 32;
+    float xt[N], xd[N], w[N];
+#pragma unroll
+    for (int k = 0; k < N; ++k) xd[k] = 0.f;
+    // fp64 prefix over slabs: each lane owns a contiguous run of slabs
+    const int per = (nslab + 31) / 32;
+    const int s0 = min(lane * per, nslab), s1 = min(s0 + per, nslab);
+    double mine = 0.0;
+    for (int s = s0; s < s1; ++s) mine += (double)slab_sum[s];
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    const double total = __shfl_sync(0xffffffffu, incl, 31);
+    const double tau = (double)u01 * total;
+    // first slab whose inclusive prefix exceeds tau
+    double run = incl - mine;
+    int found = -1;
+    double base = 0.0;
+    for (int s = s0; s < s1; ++s) {
+        const double nxt = run + (double)slab_sum[s];
+        if (found < 0 && nxt > tau) { found = s; base = run; }
+        run = nxt;
+    }
+    const unsigned m = __ballot_sync(0xffffffffu, found >= 0);
+    int slab;
+    if (m) {
+        const int src = __ffs(m) - 1;
+        slab = __shfl_sync(0xffffffffu, found, src);
+        base = __shfl_sync(0xffffffffu, base, src);
+    } else {
+        // rounding left nothing above tau: take the last slab with positive mass
+        int lastpos = -1;
+        double lb = 0.0;
+        run = incl - mine;
+        for (int s = s0; s < s1; ++s) {
+            if (slab_sum[s] > 0.f) { lastpos = s; lb = run; }
+            run += (double)slab_sum[s];
+        }
+        const unsigned pm = __ballot_sync(0xffffffffu, lastpos >= 0);
+        const int src = pm ? 31 - __clz(pm) : 0;
+        slab = __shfl_sync(0xffffffffu, lastpos, src);
+        base = __shfl_sync(0xffffffffu, lb, src);
+        if (slab < 0) { slab = 0; base = 0.0; }
+    }
+    // walk inside the slab
+    const int j = slab * 32 + lane;
+    float ls = 0.f;
+#pragma unroll
+    for (int k = 0; k < N; ++k) w[k] = 0.f;
+    if (j < nvec) {
+        load_vec<T, VEC>(trow, j, V, xt);
+        if (mode == 1) load_vec<T, VEC>(drow, j, V, xd);
+        ls = vec_weights<N>(xt, xd, P.c, np, nq, mode, w);
+    }
+    float li = ls;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float up = __shfl_up_sync(0xffffffffu, li, o);
+        if (lane >= o) li += up;
+    }
+    float lex = __shfl_up_sync(0xffffffffu, li, 1);
+    if (lane == 0) lex = 0.f;
+    const unsigned hm = __ballot_sync(0xffffffffu, base + (double)li > tau);
+    const unsigned pm = __ballot_sync(0xffffffffu, ls > 0.f);
+    const int sel = hm ? __ffs(hm) - 1 : (pm ? 31 - __clz(pm) : -1);
+    int tok = min(slab * 32 * N, V - 1);
+    if (sel >= 0 && lane == sel) {
+        double acc = base + (double)lex;
+        int pick = -1, lastp = 0;
+#pragma unroll
+        for (int k = 0; k < N; ++k) {
+            acc += (double)w[k];
+            if (w[k] > 0.f) lastp = k;
+            if (pick < 0 && acc > tau) pick = k;
+        }
+        if (pick < 0) pick = lastp;
+        tok = min(j * N + pick, V - 1);
+    }
+    if (sel >= 0) tok = __shfl_sync(0xffffffffu, tok, sel);
+    *total_out = total;
+    return tok;
 }
 
 // Block-wide inverse-CDF draw over the rows of one unit, read from global memory (L2).
@@ -229,148 +353,114 @@ __device__ void unit_draw(const VerifyParams& P, const T* __restrict__ trow, con
 #pragma unroll
     for (int k = 0; k < N; ++k) xd[k] = 0.f;
 
-    for (int s = warp; s < nslab; s += nwarp) {
-        const int j = s * 32 + lane;
-        float ls = 0.f;
-        if (j < nvec) {
-            load_vec<T, VEC>(trow, j, V, xt);
-            if (mode == 1) load_vec<T, VEC>(drow, j, V, xd);
-            ls = vec_weights<N>(xt, xd, P.c, np, nq, mode, w);
-        }
+    if constexpr (VEC) {
+        // four slabs per trip: all loads are issued before any of them is consumed
+        constexpr int U = 4;
+        const uint4* tv = reinterpret_cast<const uint4*>(trow);
+        const uint4* dv = reinterpret_cast<const uint4*>(drow);
+        for (int s0 = warp; s0 < nslab; s0 += nwarp * U) {
+            uint4 rt[U], rd[U];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
-        if (lane == 0) slab_sum[s] = ls;
+            for (int k = 0; k < U; ++k) {
+                const int j = (s0 + k * nwarp) * 32 + lane;
+                rt[k] = rd[k] = make_uint4(0, 0, 0, 0);
+                if (s0 + k * nwarp < nslab && j < nvec) {
+                    rt[k] = __ldcg(tv + j);
+                    if (mode == 1) rd[k] = __ldcg(dv + j);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                const int s = s0 + k * nwarp;
+                if (s >= nslab) break;
+                float ls = 0.f;
+                if (s * 32 + lane < nvec) {
+                    unpack(rt[k], xt);
+                    unpack(rd[k], xd);
+                    ls = vec_weights<N>(xt, xd, P.c, np, nq, mode, w);
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+                if (lane == 0) slab_sum[s] = ls;
+            }
+        }
+    } else {
+        for (int s = warp; s < nslab; s += nwarp) {
+            const int j = s * 32 + lane;
+            float ls = 0.f;
+            if (j < nvec) {
+                load_vec<T, VEC>(trow, j, V, xt);
+                if (mode == 1) load_vec<T, VEC>(drow, j, V, xd);
+                ls = vec_weights<N>(xt, xd, P.c, np, nq, mode, w);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+            if (lane == 0) slab_sum[s] = ls;
+        }
     }
     bar_sync(bar_id, nthreads);
 
     if (warp == 0) {
-        // fp64 prefix over slabs: each lane owns a contiguous run of slabs
-        const int per = (nslab + 31) / 32;
-        const int s0 = min(lane * per, nslab), s1 = min(s0 + per, nslab);
-        double mine = 0.0;
-        for (int s = s0; s < s1; ++s) mine += (double)slab_sum[s];
-        double incl = mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const double up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
-        }
-        const double total = __shfl_sync(0xffffffffu, incl, 31);
-        const double tau = (double)u01 * total;
-        // first slab whose inclusive prefix exceeds tau
-        double run = incl - mine;
-        int found = -1;
-        double base = 0.0;
-        for (int s = s0; s < s1; ++s) {
-            const double nxt = run + (double)slab_sum[s];
-            if (found < 0 && nxt > tau) { found = s; base = run; }
-            run = nxt;
-        }
-        const unsigned m = __ballot_sync(0xffffffffu, found >= 0);
-        int slab;
-        if (m) {
-            const int src = __ffs(m) - 1;
-            slab = __shfl_sync(0xffffffffu, found, src);
-            base = __shfl_sync(0xffffffffu, base, src);
-        } else {
-            // rounding left nothing above tau: take the last slab with positive mass
-            int lastpos = -1;
-            double lb = 0.0;
-            run = incl - mine;
-            for (int s = s0; s < s1; ++s) {
-                if (slab_sum[s] > 0.f) { lastpos = s; lb = run; }
-                run += (double)slab_sum[s];
-            }
-            const unsigned pm = __ballot_sync(0xffffffffu, lastpos >= 0);
-            const int src = pm ? 31 - __clz(pm) : 0;
-            slab = __shfl_sync(0xffffffffu, lastpos, src);
-            base = __shfl_sync(0xffffffffu, lb, src);
-            if (slab < 0) { slab = 0; base = 0.0; }
-        }
-        // walk inside the slab
-        const int j = slab * 32 + lane;
-        float ls = 0.f;
-#pragma unroll
-        for (int k = 0; k < N; ++k) w[k] = 0.f;
-        if (j < nvec) {
-            load_vec<T, VEC>(trow, j, V, xt);
-            if (mode == 1) load_vec<T, VEC>(drow, j, V, xd);
-            ls = vec_weights<N>(xt, xd, P.c, np, nq, mode, w);
-        }
-        float li = ls;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float up = __shfl_up_sync(0xffffffffu, li, o);
-            if (lane >= o) li += up;
-        }
-        float lex = __shfl_up_sync(0xffffffffu, li, 1);
-        if (lane == 0) lex = 0.f;
-        const unsigned hm = __ballot_sync(0xffffffffu, base + (double)li > tau);
-        const unsigned pm = __ballot_sync(0xffffffffu, ls > 0.f);
-        const int sel = hm ? __ffs(hm) - 1 : (pm ? 31 - __clz(pm) : -1);
-        int tok = min(slab * 32 * N, V - 1);
-        if (sel >= 0 && lane == sel) {
-            double acc = base + (double)lex;
-            int pick = -1, lastp = 0;
-#pragma unroll
-            for (int k = 0; k < N; ++k) {
-                acc += (double)w[k];
-                if (w[k] > 0.f) lastp = k;
-                if (pick < 0 && acc > tau) pick = k;
-            }
-            if (pick < 0) pick = lastp;
-            tok = min(j * N + pick, V - 1);
-        }
-        if (sel >= 0) tok = __shfl_sync(0xffffffffu, tok, sel);
+        double total;
+        const int tok = draw_select<T, VEC>(P, trow, drow, mode, u01, np, nq, slab_sum, lane, &total);
         if (lane == 0) { sh.token = tok; sh.total = total; }
     }
     bar_sync(bar_id, nthreads);
 }
 
-// Row bookkeeping by one full warp of a unit after its (optional) draw: record the draw, count
-// the arrival, and let the last position of the row to arrive resolve n and y' (warp ballot
-// over the accept flags of positions < L).
-__device__ __forceinline__ void unit_finish(const VerifyParams& P, const Unit& u, int have_draw, int token, float mass,
-                                            int lane) {
-    const int K = P.K;
+// Row bookkeeping, by one full warp of a unit.  row_arrive counts the unit on its row and tells
+// whether it was the row's last; row_resolve (last arriver only) ballots the accept flags of the
+// positions < L into n = first rejection (or L) and reports bad tokens.
+__device__ __forceinline__ bool row_arrive(const VerifyParams& P, const Unit& u, int lane) {
     int last = 0;
-    if (lane == 0) {
-        P.draws[(size_t)u.b * (K + 1) + u.i] = have_draw ? token : -1;
-        P.draw_mass[(size_t)u.b * (K + 1) + u.i] = mass;
-        __threadfence();
-        const int old = atomicAdd(&P.arrive[u.b], 1);
-        last = (old == u.L);
-        if (last) __threadfence();
-    }
-    last = __shfl_sync(0xffffffffu, last, 0);
-    if (!last) return;
-    int n = u.L, bad = 0;
+    // release: this unit's flag (and draw) are visible before the count; acquire: the last
+    // arriver sees every other unit's
+    if (lane == 0) last = (atom_add_acq_rel(&P.arrive[u.b], 1) == u.L);
+    return __shfl_sync(0xffffffffu, last, 0) != 0;
+}
+__device__ __forceinline__ void row_resolve(const VerifyParams& P, const Unit& u, int lane, int& n, int& bad) {
+    n = u.L;
+    bad = 0;
     for (int j0 = 0; j0 < u.L; j0 += 32) {
         const int j = j0 + lane;
         int st = FLAG_ACCEPT;
-        if (j < u.L) st = ld_acquire(&P.flags[(size_t)u.b * K + j]) & 3;
+        if (j < u.L) st = ld_acquire(&P.flags[(size_t)u.b * P.K + j]) & 3;
         const unsigned rej = __ballot_sync(0xffffffffu, st >= FLAG_REJECT);
         const unsigned bd = __ballot_sync(0xffffffffu, st == FLAG_BAD);
         if (rej && n == u.L) n = j0 + __ffs(rej) - 1;
         bad |= (bd != 0);
     }
+    if (lane == 0) P.arrive[u.b] = 0;               // ready for the next call
+    // positions the method never looks at report zeros
+    if (P.ratio)
+        for (int j = u.L + lane; j < P.K; j += 32) P.ratio[(size_t)u.b * P.K + j] = 0.f;
+    if (P.stats)
+        for (int j = (u.L + 1) * 4 + lane; j < (P.K + 1) * 4; j += 32) P.stats[(size_t)u.b * (P.K + 1) * 4 + j] = 0.f;
+}
+
+// For kernels that draw inside the unit: record the draw, count the arrival, and let the last
+// position of the row to arrive pick n and the draw made at position n.
+__device__ __forceinline__ void unit_finish(const VerifyParams& P, const Unit& u, int have_draw, int token, float mass,
+                                            int lane) {
+    const int K = P.K;
+    if (lane == 0 && have_draw) {
+        st_relaxed(&P.draws[(size_t)u.b * (K + 1) + u.i], token);
+        st_relaxed(reinterpret_cast<int32_t*>(&P.draw_mass[(size_t)u.b * (K + 1) + u.i]), __float_as_int(mass));
+    }
+    if (!row_arrive(P, u, lane)) return;
+    int n, bad;
+    row_resolve(P, u, lane, n, bad);
     if (lane == 0) {
         int tok = -1;
         float m = 0.f;
         if (!bad) {
             tok = ld_acquire(&P.draws[(size_t)u.b * (K + 1) + n]);
-            m = __ldcg(&P.draw_mass[(size_t)u.b * (K + 1) + n]);
+            m = __int_as_float(ld_acquire(reinterpret_cast<const int32_t*>(&P.draw_mass[(size_t)u.b * (K + 1) + n])));
         }
         P.n_acc[u.b] = bad ? -1 : n;
         P.next[u.b] = tok;
         if (P.rmass) P.rmass[u.b] = bad ? 0.f : (n == u.L ? 1.f : m);
-        P.arrive[u.b] = 0;                      // ready for the next call
     }
-    // positions the method never looks at report zeros
-    if (P.ratio)
-        for (int j = u.L + lane; j < K; j += 32) P.ratio[(size_t)u.b * K + j] = 0.f;
-    if (P.stats)
-        for (int j = (u.L + 1) * 4 + lane; j < (K + 1) * 4; j += 32) P.stats[(size_t)u.b * (K + 1) * 4 + j] = 0.f;
 }
 
 }  // namespace sd

@@ -81,17 +81,19 @@ __global__ void __launch_bounds__(STATIC_THREADS, 2) verify_static_kernel(const 
         Acc a = lane < NW ? sh.wp[lane] : acc_init(), b = lane < NW ? sh.wq[lane] : acc_init();
         a = warp_merge(a);
         b = warp_merge(b);
+        int y = 0, y_ok = 1;
+        float t_y = 0.f, d_y = 0.f, r = 0.f;
+        if (lane == 0 && !u.bonus) {
+            r = P.uniforms[(size_t)u.b * (P.K + 1) + u.i];
+            y = P.tokens[(size_t)u.b * P.K + u.i];
+            y_ok = (y >= 0 && y < P.V);
+            if (y_ok) { t_y = to_float(trow[y]); d_y = to_float(drow[y]); }
+        }
+        const int mode = unit_decide(P, u, a, b, t_y, d_y, y_ok, r, lane);
         if (lane == 0) {
-            int y = 0, y_ok = 1;
-            float t_y = 0.f, d_y = 0.f;
-            if (!u.bonus) {
-                y = P.tokens[(size_t)u.b * P.K + u.i];
-                y_ok = (y >= 0 && y < P.V);
-                if (y_ok) { t_y = to_float(trow[y]); d_y = to_float(drow[y]); }
-            }
             sh.np = make_norm(a);
             sh.nq = u.bonus ? sh.np : make_norm(b);
-            sh.need_draw = unit_decide(P, u, a, b, t_y, d_y, y_ok);
+            sh.need_draw = mode;
         }
     }
     __syncthreads();
@@ -203,6 +205,9 @@ extern "C" int specdec_verify_correct_static(const void* target_logits, const vo
     p.draw_mass = reinterpret_cast<float*>(base + OFF_MASS);
     p.arrive = reinterpret_cast<int32_t*>(base + OFF_ARRIVE);
     p.status = data_status ? data_status : reinterpret_cast<uint32_t*>(base + OFF_STATUS);
+    p.norms = nullptr;
+    p.tasks = nullptr;
+    p.task_ctl = nullptr;
     p.epoch = epoch;
     e = dtype == SPECDEC_BF16 ? launch_static<__nv_bfloat16>(p, s) : launch_static<float>(p, s);
     if (e != cudaSuccess)
