@@ -1,10 +1,355 @@
-// Acceptance-prediction head (Eq. 3 / Section 5.1 of arXiv 2405.19715).
+// Acceptance-prediction head (Eq. 3 and Section 5.1 of arXiv 2405.19715):
+//   x_k = x_{k-1} + SiLU(W_k x_{k-1} + b_k), k = 1..D;  accept_prob = sigmoid(w_out . x_D + b_out).
+//
+// Each residual block is one GEMM  Z[M, d] = X[M, d] * W^T  (W stored [out, in], so both operands
+// are K-major) on the 5th-generation tensor cores: operand tiles arrive in shared memory by TMA
+// (128-byte swizzle), one thread issues tcgen05.mma with the fp32 accumulator in tensor memory,
+// and four epilogue warps read the accumulator back with tcgen05.ld and apply bias, SiLU and
+// the residual.  The last block does not store x_D: its epilogue multiplies by w_out and leaves
+// one partial dot product per (row, column tile); a small kernel adds them and applies the
+// sigmoid.  D = 0 is a plain row-times-vector kernel.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
 #include <cstdio>
 
 #include "specdec_internal.h"
 
-extern "C" int specdec_accept_head(specdec_ctx* ctx, const void*, const specdec_head*, int, int, float*, void*) {
+namespace {
+
+constexpr int BM = 128;                  // rows of X per CTA (= UMMA M)
+constexpr int BK = 64;                   // bf16 elements per k-block: one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr int HEAD_THREADS = 192;        // warp 0 TMA, warp 1 MMA + tensor-memory owner, warps 2..5 epilogue
+constexpr uint32_t WAIT_POLLS = 1u << 24;
+
+template <int BN> struct Cfg {
+    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int A_BYTES = BM * BK * 2;
+    static constexpr int B_BYTES = BN * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: on exhaustion a status bit is set and execution simply continues, so every
+// thread still reaches the barriers and the tensor-memory release below.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status) {
+    for (uint32_t it = 0; it < WAIT_POLLS; ++it)
+        if (mbar_try_wait(bar, parity)) return;
+    atomicOr(status, SPECDEC_DATA_WAIT_LIMIT);
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled:
+// start address, leading offset 16 B (unused by swizzled layouts), 1024 B between 8-row groups,
+// descriptor version 1, layout type SWIZZLE_128B.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+    return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t umma_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ float silu(float z) { return __fdividef(z, 1.f + __expf(-z)); }
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+struct BlockParams {
+    const __nv_bfloat16* X;      // [M, d] input of the block (also the residual)
+    const __nv_bfloat16* bias;   // [d] or null
+    __nv_bfloat16* Y;            // [M, d] output, null for the last block
+    const __nv_bfloat16* w_out;  // [d], last block only
+    float* partial;              // [M, d / BN], last block only
+    int M, d;
+    uint32_t* status;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(HEAD_THREADS, 1)
+head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
+                  const BlockParams P) {
+    using C = Cfg<BN>;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
+    unsigned char* aligned = smem_raw + (base - smem_u32(smem_raw));
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(aligned + C::STAGES * C::STAGE_BYTES);
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * C::STAGES, tfull = empty0 + 8 * C::STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int nkb = P.d / BK;
+
+    if (tid == 0) {
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(tfull, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {                      // this warp owns the tensor-memory allocation
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            for (int kb = 0; kb < nkb; ++kb) {
+                mbar_wait(empty0 + 8 * stage, phase ^ 1u, P.status);
+                const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
+                mbar_expect_tx(full0 + 8 * stage, C::STAGE_BYTES);
+                tma_load_2d(a, &mapX, kb * BK, m0, full0 + 8 * stage);
+                tma_load_2d(b, &mapW, kb * BK, n0, full0 + 8 * stage);
+                if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc(BN);
+            uint32_t stage = 0, phase = 0;
+            for (int kb = 0; kb < nkb; ++kb) {
+                mbar_wait(full0 + 8 * stage, phase, P.status);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k)
+                    umma_bf16(tmem, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), idesc,
+                              (kb | k) != 0 ? 1u : 0u);
+                umma_commit(empty0 + 8 * stage);          // stage reusable once these MMAs have read it
+                if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+            }
+            umma_commit(tfull);                            // accumulator complete
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps
+        const int q = warp & 3;                            // tensor-memory lane quarter this warp may read
+        const int m = m0 + q * 32 + lane;
+        const bool row_ok = m < P.M;
+        mbar_wait(tfull, 0, P.status);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint4* xrow = reinterpret_cast<const uint4*>(P.X + (size_t)(row_ok ? m : 0) * P.d + n0);
+        float dot = 0.f;
+#pragma unroll 1
+        for (int c = 0; c < BN / 32; ++c) {
+            float acc[32];
+            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), acc);
+            uint4 xv[4], bv[4], wv[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                xv[j] = row_ok ? __ldg(xrow + c * 4 + j) : make_uint4(0, 0, 0, 0);
+                bv[j] = P.bias ? __ldg(reinterpret_cast<const uint4*>(P.bias + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
+                wv[j] = P.w_out ? __ldg(reinterpret_cast<const uint4*>(P.w_out + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
+            }
+            const uint32_t* xw = reinterpret_cast<const uint32_t*>(xv);
+            const uint32_t* bw = reinterpret_cast<const uint32_t*>(bv);
+            const uint32_t* ww = reinterpret_cast<const uint32_t*>(wv);
+            uint32_t out[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const float y0 = bf16lo(xw[j]) + silu(acc[2 * j] + bf16lo(bw[j]));
+                const float y1 = bf16hi(xw[j]) + silu(acc[2 * j + 1] + bf16hi(bw[j]));
+                dot = fmaf(y0, bf16lo(ww[j]), dot);
+                dot = fmaf(y1, bf16hi(ww[j]), dot);
+                const __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
+                out[j] = *reinterpret_cast<const uint32_t*>(&pk);
+            }
+            if (P.Y && row_ok) {
+                uint4* yrow = reinterpret_cast<uint4*>(P.Y + (size_t)m * P.d + n0 + c * 32);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) yrow[j] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+            }
+        }
+        if (P.partial && row_ok) P.partial[(size_t)m * gridDim.x + blockIdx.x] = dot;
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
+    }
+}
+
+// accept_prob[m] = sigmoid(sum_t partial[m, t] + b_out)
+__global__ void head_finish_kernel(const float* __restrict__ partial, int M, int nt, float b_out,
+                                   float* __restrict__ accept_prob) {
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= M) return;
+    float s = b_out;
+    for (int t = 0; t < nt; ++t) s += partial[(size_t)m * nt + t];
+    accept_prob[m] = 1.f / (1.f + __expf(-s));
+}
+
+// D = 0: one warp per row, accept_prob[m] = sigmoid(hidden[m, :] . w_out + b_out)
+__global__ void head_linear_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ w, int M,
+                                   int d, float b_out, float* __restrict__ accept_prob) {
+    const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (m >= M) return;
+    const uint4* xr = reinterpret_cast<const uint4*>(X + (size_t)m * d);
+    const uint4* wr = reinterpret_cast<const uint4*>(w);
+    float s = 0.f;
+    for (int v = lane; v < d / 8; v += 32) {
+        const uint4 a = __ldg(xr + v), b = __ldg(wr + v);
+        const uint32_t* aw = reinterpret_cast<const uint32_t*>(&a);
+        const uint32_t* bw = reinterpret_cast<const uint32_t*>(&b);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) s = fmaf(bf16lo(aw[j]), bf16lo(bw[j]), fmaf(bf16hi(aw[j]), bf16hi(bw[j]), s));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) accept_prob[m] = 1.f / (1.f + __expf(-(s + b_out)));
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// 2-D bf16 row-major [rows, cols] tensor, box {BK, box_rows}, 128-byte swizzle, zero fill outside.
+bool make_map(CUtensorMap* map, const void* ptr, int rows, int cols, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+cudaError_t launch_block(const CUtensorMap& mx, const CUtensorMap& mw, const BlockParams& p, cudaStream_t s) {
+    cudaError_t e = cudaFuncSetAttribute(head_block_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM);
+    if (e != cudaSuccess) return e;
+    dim3 grid(p.d / BN, (p.M + BM - 1) / BM);
+    head_block_kernel<BN><<<grid, HEAD_THREADS, Cfg<BN>::SMEM, s>>>(mx, mw, p);
+    return cudaGetLastError();
+}
+
+int fail(specdec_ctx* ctx, int code, const char* msg) {
+    snprintf(ctx->err, sizeof(ctx->err), "%s", msg);
+    return code;
+}
+
+}  // namespace
+
+extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const specdec_head* head, int B, int K,
+                                   float* accept_prob, void* stream) {
     if (!ctx) return SPECDEC_EINVAL;
-    snprintf(ctx->err, sizeof(ctx->err), "accept_head: not built yet");
-    return SPECDEC_EUNSUPPORTED;
+    if (!hidden || !head || !accept_prob || !head->w_out) return fail(ctx, SPECDEC_EINVAL, "accept_head: null pointer argument");
+    if (B < 1 || K < 1) return fail(ctx, SPECDEC_EINVAL, "accept_head: B and K must be >= 1");
+    const int d = head->d, D = head->depth;
+    if (D < 0 || D > 8) return fail(ctx, SPECDEC_EINVAL, "accept_head: depth must be in [0, 8]");
+    if (D > 0 && !head->W) return fail(ctx, SPECDEC_EINVAL, "accept_head: null weight list");
+    if (d < 128 || d % 128 != 0) return fail(ctx, SPECDEC_EUNSUPPORTED, "accept_head: d must be a positive multiple of 128");
+    const long long M = (long long)B * K;
+    if (d > ctx->max_d || M > (long long)ctx->max_B * ctx->max_K)
+        return fail(ctx, SPECDEC_EUNSUPPORTED, "accept_head: B*K or d exceed the context");
+    if (reinterpret_cast<uintptr_t>(hidden) % 16 != 0 || reinterpret_cast<uintptr_t>(head->w_out) % 16 != 0)
+        return fail(ctx, SPECDEC_EINVAL, "accept_head: hidden and w_out must be 16-byte aligned");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(hidden);
+    if (D == 0) {
+        const int wpb = 8;
+        head_linear_kernel<<<(int)((M + wpb - 1) / wpb), wpb * 32, 0, s>>>(x, static_cast<const __nv_bfloat16*>(head->w_out),
+                                                                            (int)M, d, head->b_out, accept_prob);
+        ctx->launches += 1;
+        cudaError_t e = cudaGetLastError();
+        return e == cudaSuccess ? SPECDEC_OK : fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
+    }
+    const int BN = d % 256 == 0 ? 256 : 128;
+    for (int k = 0; k < D; ++k) {
+        const void* W = head->W[k];
+        const void* bias = head->b ? head->b[k] : nullptr;
+        if (!W || reinterpret_cast<uintptr_t>(W) % 16 != 0 || (bias && reinterpret_cast<uintptr_t>(bias) % 16 != 0))
+            return fail(ctx, SPECDEC_EINVAL, "accept_head: weights and biases must be non-null and 16-byte aligned");
+        const bool last = (k == D - 1);
+        CUtensorMap mx, mw;
+        if (!make_map(&mx, x, (int)M, d, BM) || !make_map(&mw, W, d, d, BN))
+            return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
+        BlockParams p;
+        p.X = x;
+        p.bias = static_cast<const __nv_bfloat16*>(bias);
+        p.Y = last ? nullptr : static_cast<__nv_bfloat16*>(ctx->act[k & 1]);
+        p.w_out = last ? static_cast<const __nv_bfloat16*>(head->w_out) : nullptr;
+        p.partial = last ? ctx->head_partial : nullptr;
+        p.M = (int)M;
+        p.d = d;
+        p.status = ctx->status;
+        cudaError_t e = BN == 256 ? launch_block<256>(mx, mw, p, s) : launch_block<128>(mx, mw, p, s);
+        if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
+        ctx->launches += 1;
+        x = p.Y;
+    }
+    head_finish_kernel<<<(int)((M + 127) / 128), 128, 0, s>>>(ctx->head_partial, (int)M, d / BN, head->b_out, accept_prob);
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? SPECDEC_OK : fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
 }

@@ -80,15 +80,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar, uint32_t parity, uint32_t ns) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
-    return ok != 0;
-}
 // Bounded wait.  A wait that runs out records SPECDEC_DATA_WAIT_LIMIT and returns; control flow
 // never depends on it, so no thread can be left behind at a barrier (outputs are then invalid).
 __device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status) {
@@ -107,11 +98,7 @@ __device__ __forceinline__ void mbar_wait_warp(uint32_t bar, uint32_t parity, ui
 __device__ __forceinline__ void mbar_wait_relaxed(uint32_t bar, uint32_t parity, uint32_t* status, int lane) {
     if (lane == 0) {
         bool ok = false;
-#ifdef EXP_HINT
-        for (uint32_t it = 0; it < WAIT_POLLS && !(ok = mbar_try_wait_hint(bar, parity, 20000u)); ++it) {}
-#else
         for (uint32_t it = 0; it < WAIT_POLLS && !(ok = mbar_try_wait(bar, parity)); ++it) __nanosleep(256);
-#endif
         if (!ok) atomicOr(status, SPECDEC_DATA_WAIT_LIMIT);
     }
     __syncwarp();
@@ -276,11 +263,7 @@ __device__ __forceinline__ void produce_unit(StreamShared& ss, uint32_t ring, co
         const uint32_t off = (uint32_t)t * TILE_BYTES;
         const uint32_t bytes = min((uint32_t)TILE_BYTES, row_bytes - off);
         const uint32_t full = smem_u32(&ss.full[stage]);
-#ifdef EXP_HINT
-        { bool ok = false; for (uint32_t it = 0; it < WAIT_POLLS && !(ok = mbar_try_wait_hint(smem_u32(&ss.empty[stage]), phase ^ 1u, 20000u)); ++it) {} if (!ok) atomicOr(status, SPECDEC_DATA_WAIT_LIMIT); }
-#else
         mbar_wait(smem_u32(&ss.empty[stage]), phase ^ 1u, status);
-#endif
         mbar_expect_tx(full, single ? bytes : 2 * bytes);
         const uint32_t dst = ring + stage * (2 * TILE_BYTES);
         bulk_load(dst, tsrc + off, bytes, full);

@@ -1,0 +1,102 @@
+"""GPU parity of specdec_accept_head (tcgen05 GEMMs) and of the head -> stop -> verify chain of
+cfg5 against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from oracle import specdec_oracle as orc  # noqa: E402
+from paper_2405_19715_b200 import specdec, workloads as wl  # noqa: E402
+from tests import parity  # noqa: E402
+
+HEAD_RTOL = 2e-2      # spec tolerance for bf16 head outputs
+
+
+def _head_problem(seed, B, K, d, depth, with_bias, std=0.05):
+    rng = np.random.default_rng(seed)
+    hidden = wl.f32_to_bf16_bits(rng.standard_normal((B, K, d), dtype=np.float32))
+    Ws = [wl.f32_to_bf16_bits((rng.standard_normal((d, d), dtype=np.float32) * std)) for _ in range(depth)]
+    bs = [wl.f32_to_bf16_bits(rng.standard_normal(d, dtype=np.float32) * 0.3) if with_bias else None for _ in range(depth)]
+    w_out = wl.f32_to_bf16_bits(rng.standard_normal(d, dtype=np.float32) * std)
+    return hidden, Ws, bs, w_out, float(rng.normal() * 0.2)
+
+
+def _run_head(ctx, hidden, Ws, bs, w_out, b_out):
+    th = specdec.from_numpy(hidden)
+    tW = [specdec.from_numpy(w) for w in Ws]
+    tb = [None if b is None else specdec.from_numpy(b) for b in bs]
+    out = specdec.specdec_accept_head(ctx, th, tW, tb, specdec.from_numpy(w_out), b_out)
+    torch.cuda.synchronize()
+    assert ctx.device_status() == 0
+    return out.cpu().numpy()
+
+
+@pytest.mark.parametrize("d", [128, 256, 384, 512])
+@pytest.mark.parametrize("depth", [0, 1, 2, 3])
+@pytest.mark.parametrize("with_bias", [False, True])
+def test_head_small_shapes(d, depth, with_bias):
+    B, K = 7, 23                      # 161 rows: one full 128-row tile and a ragged one
+    ctx = specdec.Context(B, K, max_d=d)
+    hidden, Ws, bs, w_out, b_out = _head_problem(100 + d + depth, B, K, d, depth, with_bias)
+    got = _run_head(ctx, hidden, Ws, bs, w_out, b_out)
+    want = orc.accept_head(hidden, list(zip(Ws, bs)), w_out, b_out)
+    err = np.abs(got - want) / want
+    assert err.max() <= HEAD_RTOL, (err.max(), got.ravel()[:4], want.ravel()[:4])
+    # a transposed or mis-tiled operand would be off by far more than the tolerance; make sure the
+    # outputs are not degenerate either
+    assert want.std() > 1e-3
+    ctx.close()
+
+
+def test_head_reduces_to_logistic_regression_when_weights_are_zero():
+    B, K, d = 4, 40, 256
+    ctx = specdec.Context(B, K, max_d=d)
+    hidden, Ws, bs, w_out, b_out = _head_problem(5, B, K, d, 2, False)
+    Ws = [np.zeros_like(w) for w in Ws]
+    got = _run_head(ctx, hidden, Ws, bs, w_out, b_out)
+    want = orc.accept_head(hidden, [], w_out, b_out)
+    np.testing.assert_allclose(got, want, rtol=1e-4)
+    ctx.close()
+
+
+def test_head_argument_errors():
+    ctx = specdec.Context(4, 4, max_d=256)
+    h = torch.zeros(4, 4, 192, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(192, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(specdec.SpecdecError) as e:
+        specdec.specdec_accept_head(ctx, h, [], None, w, 0.0)
+    assert e.value.code == specdec.EUNSUPPORTED
+    h = torch.zeros(4, 4, 512, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(specdec.SpecdecError) as e:
+        specdec.specdec_accept_head(ctx, h, [], None, torch.zeros(512, dtype=torch.bfloat16, device="cuda"), 0.0)
+    assert e.value.code == specdec.EUNSUPPORTED
+    ctx.close()
+
+
+def test_config5_head_stop_verify_chain():
+    """cfg5: hidden [128,16,4096] -> D=2 head -> stop at h=0.5 -> cand_len = min(stop_pos + 2, K)
+    -> verify/correct at V=32000 (bf16, T=0.7)."""
+    cfg = wl.CONFIGS["cfg5"]
+    ctx = specdec.Context(cfg.B, cfg.K, max_d=cfg.d)
+    hd = wl.make_head_inputs(cfg)
+    Ws = [w for w, _ in hd["blocks"]]
+    bs = [b for _, b in hd["blocks"]]
+    got = _run_head(ctx, hd["hidden"], Ws, bs, hd["w_out"], float(hd["b_out"]))
+    want = orc.accept_head(hd["hidden"], hd["blocks"], hd["w_out"], float(hd["b_out"]))
+    err = np.abs(got - want) / want
+    print("cfg5 head max rel err", err.max())
+    assert err.max() <= HEAD_RTOL
+    # stop rule on the GPU's own probabilities (same inputs on both sides)
+    pos = specdec.specdec_stop(ctx, torch.from_numpy(got).cuda(), cfg.h).cpu().numpy()
+    rep = parity.classify_stop(got, cfg.h, pos)
+    assert rep["exact"] + rep["boundary"] == cfg.B
+    cand_len = np.minimum(pos + 2, cfg.K).astype(np.int32)     # Algorithm 1: one more token was drafted
+    print("cfg5 cand_len histogram", np.bincount(cand_len, minlength=cfg.K + 1).tolist())
+    inp = wl.make_verify_inputs(cfg)
+    inp["cand_len"] = cand_len
+    gpu = parity.run_gpu_verify(ctx, inp)
+    rep = parity.classify_rows(inp, gpu, dtype="f32")
+    print("cfg5 verify", rep)
+    assert ctx.device_status() == 0
+    ctx.close()
