@@ -131,7 +131,7 @@ def algorithmic_bytes(cfg: wl.Workload, lens: np.ndarray) -> int:
 
 
 # ----------------------------------------------------------------------------------------- CPU arm
-def oracle_sample_rate(cfg: wl.Workload, inp: dict, budget_s: float, accept_prob=None):
+def oracle_sample_rate(cfg: wl.Workload, inp: dict, budget_s: float, head=None):
     """Times the CPU oracle (as it stands) on leading batch rows until `budget_s` is used.
     Returns (tokens/s, rows used, seconds, threads)."""
     from oracle import specdec_oracle as orc
@@ -141,8 +141,9 @@ def oracle_sample_rate(cfg: wl.Workload, inp: dict, budget_s: float, accept_prob
     chunk = 4
     while rows < cfg.B and time.perf_counter() - t0 < budget_s:
         sl = slice(rows, min(rows + chunk, cfg.B))
-        if accept_prob is not None:
-            orc.stop_rule(accept_prob[sl], cfg.h, lens[sl])
+        if head is not None:
+            a = orc.accept_head(head["hidden"][sl], head["blocks"], head["w_out"], float(head["b_out"]))
+            orc.stop_rule(a.astype(np.float32), cfg.h, lens[sl])
         orc.verify_correct(inp["target_logits"][sl], inp["draft_logits"][sl], inp["cand_tokens"][sl], lens[sl],
                            inp["uniforms"][sl], inp["temperature"])
         tokens += int(lens[sl].sum())
@@ -157,12 +158,13 @@ def run_reference(args, cfg):
         return
     sub = cfg.scaled(B=min(cfg.B, 8))          # bounded sample: the first rows of the workload
     inp = wl.make_verify_inputs(sub)
-    a = wl.make_accept_prob(sub)
+    hd = wl.make_head_inputs(wl.CONFIGS["cfg5"].scaled(B=sub.B, K=sub.K, seed=sub.seed))
     rates = []
     for it in range(args.warmup + args.steps):
         t0 = time.perf_counter()
         from oracle import specdec_oracle as orc
-        orc.stop_rule(a, sub.h, inp["cand_len"])
+        a = orc.accept_head(hd["hidden"], hd["blocks"], hd["w_out"], float(hd["b_out"]))
+        orc.stop_rule(a.astype(np.float32), sub.h, inp["cand_len"])
         orc.verify_correct(inp["target_logits"], inp["draft_logits"], inp["cand_tokens"], inp["cand_len"],
                            inp["uniforms"], inp["temperature"])
         dt = time.perf_counter() - t0
@@ -183,8 +185,8 @@ def run_reference(args, cfg):
 
 
 def workload_config(cfg: wl.Workload, world: int) -> dict:
-    return {"workload": f"{cfg.name}: stop rule + verify/correct, B={cfg.B} K={cfg.K} V={cfg.V} {cfg.dtype} "
-                        f"T={cfg.T} (per GPU)",
+    return {"workload": f"{cfg.name}: acceptance head (d=4096, D=2) on B*K positions -> stop rule -> verify/correct, "
+                        f"B={cfg.B} K={cfg.K} V={cfg.V} {cfg.dtype} T={cfg.T} (per GPU)",
             "B_per_gpu": cfg.B, "K": cfg.K, "V": cfg.V, "logit_dtype": cfg.dtype, "sharding": f"batch rows x{world}",
             "l2": "inputs exceed L2 (no flush needed)" if cfg.B * (2 * cfg.K + 1) * cfg.V * 2 > 2 * 126e6
                   else "rotating input copies > 2x L2"}
@@ -203,7 +205,6 @@ def run_ours(args, cfg):
     cfg = cfg.scaled(seed=cfg.seed + rank)          # each rank owns its own batch rows
     inp = wl.make_verify_inputs(cfg)
     lens_np = inp["cand_len"]
-    accept_np = wl.make_accept_prob(cfg)
     es = 2 if cfg.dtype == "bf16" else 4
     per_copy = cfg.B * (2 * cfg.K + 1) * cfg.V * es
     copies = 1 if per_copy > 2 * 126e6 else int(np.ceil(2 * 126e6 / per_copy)) + 1
@@ -211,8 +212,15 @@ def run_ours(args, cfg):
     host = {k: to_torch(np.ascontiguousarray(inp[k]), "cpu", pin=True)
             for k in ("target_logits", "draft_logits", "cand_tokens", "cand_len", "uniforms")}
     devs = [{k: v.to(dev) for k, v in host.items()} for _ in range(copies)]
-    accept = torch.from_numpy(accept_np).to(dev)
-    ctx = specdec.Context(cfg.B, cfg.K)
+    # acceptance head of the cfg5 recipe (d = 4096, D = 2, N(0, 0.02^2) weights) on this batch's B x K positions
+    hcfg = wl.CONFIGS["cfg5"].scaled(B=cfg.B, K=cfg.K, seed=cfg.seed)
+    hd = wl.make_head_inputs(hcfg)
+    hidden = to_torch(hd["hidden"]).to(dev)
+    Ws = [to_torch(w).to(dev) for w, _ in hd["blocks"]]
+    bs = [to_torch(b).to(dev) for _, b in hd["blocks"]]
+    w_out = to_torch(hd["w_out"]).to(dev)
+    head_prob = torch.empty(cfg.B, cfg.K, dtype=torch.float32, device=dev)
+    ctx = specdec.Context(cfg.B, cfg.K, max_d=hcfg.d)
     n_out = torch.empty(cfg.B, dtype=torch.int32, device=dev)
     t_out = torch.empty(cfg.B, dtype=torch.int32, device=dev)
     stop_pos = torch.empty(cfg.B, dtype=torch.int32, device=dev)
@@ -220,7 +228,12 @@ def run_ours(args, cfg):
 
     def step(i, ev=None):
         d = devs[i % copies]
-        specdec.specdec_stop(ctx, accept, cfg.h, d["cand_len"], stop_pos)
+        if ev:
+            ev[2].record()
+        specdec.specdec_accept_head(ctx, hidden, Ws, bs, w_out, float(hd["b_out"]), head_prob)
+        if ev:
+            ev[3].record()
+        specdec.specdec_stop(ctx, head_prob, cfg.h, d["cand_len"], stop_pos)
         if ev:
             ev[0].record()
         specdec.specdec_verify_correct(ctx, d["target_logits"], d["draft_logits"], d["cand_tokens"], d["cand_len"],
@@ -237,7 +250,7 @@ def run_ours(args, cfg):
         sampler.start()
         time.sleep(0.2)
     launches0 = ctx.launch_count()
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    evs = [tuple(torch.cuda.Event(enable_timing=True) for _ in range(4)) for _ in range(args.steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier(world)
     torch.cuda.synchronize()
@@ -250,7 +263,9 @@ def run_ours(args, cfg):
     launches = ctx.launch_count() - launches0
     elapsed_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
     clocks = sampler.stop() if rank == 0 else None
-    verify_ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    verify_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    head_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
+    stop_ms = float(np.mean([e[3].elapsed_time(e[0]) for e in evs]))
     tokens_step = sum_over_ranks(float(lens_np.sum()), world, dev)
     ms_per_step = elapsed_ms / args.steps
     value = tokens_step / (ms_per_step * 1e-3)
@@ -259,13 +274,15 @@ def run_ours(args, cfg):
     e2e_steps = max(1, min(args.steps, 5))
     h_n = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
     h_t = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
-    h_acc = torch.from_numpy(accept_np).pin_memory()
     h_stop = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
 
+    h_hidden = to_torch(hd["hidden"], "cpu", pin=True)
+
     def e2e_step():
-        a = h_acc.to(dev, non_blocking=True)
+        hh = h_hidden.to(dev, non_blocking=True)
         l = host["cand_len"].to(dev, non_blocking=True)
-        specdec.specdec_stop(ctx, a, cfg.h, l, stop_pos)
+        specdec.specdec_accept_head(ctx, hh, Ws, bs, w_out, float(hd["b_out"]), head_prob)
+        specdec.specdec_stop(ctx, head_prob, cfg.h, l, stop_pos)
         h_stop.copy_(stop_pos, non_blocking=True)
         specdec.specdec_verify_correct_host(ctx, host["target_logits"], host["draft_logits"], host["cand_tokens"],
                                             host["cand_len"], host["uniforms"], T, h_n, h_t, flags=args.kernel)
@@ -283,13 +300,15 @@ def run_ours(args, cfg):
         e1.record()
         torch.cuda.synchronize()
         e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / e2e_steps
-    h2d = sum(v.numel() * v.element_size() for v in host.values()) + h_acc.numel() * 4 + host["cand_len"].numel() * 4
+    h2d = (sum(v.numel() * v.element_size() for v in host.values()) + h_hidden.numel() * 2
+           + host["cand_len"].numel() * 4)
     d2h = 3 * cfg.B * 4
 
     if rank != 0:
         return
     peaks = measured_peaks()
     alg = algorithmic_bytes(cfg, lens_np)
+    head_flops = 2.0 * hcfg.depth * cfg.B * cfg.K * hcfg.d * hcfg.d
     achieved = alg / (verify_ms * 1e-3) / 1e9
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
@@ -302,9 +321,14 @@ def run_ours(args, cfg):
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
                      "frac_of_nominal_8TBs": achieved / 8000.0, "algorithmic_bytes": alg, "kernel_ms": verify_ms,
                      "traffic": None},
+        "parts_ms": {"head": head_ms, "stop": stop_ms, "verify": verify_ms},
+        "roofline_head": {"kernel": "acceptance head (2 x [M,4096]x[4096,4096] bf16 GEMM)", "bound": "tensor",
+                          "achieved": head_flops / (head_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
+                          "unit": "TFLOP/s", "frac": head_flops / (head_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                          "peak_source": peaks["source"] + " cuBLAS bf16 (sustained)"},
     }
     if world == 1 and not args.no_cpu_baseline:
-        rate, rows, dt, cores = oracle_sample_rate(cfg, inp, args.cpu_budget, accept_np)
+        rate, rows, dt, cores = oracle_sample_rate(cfg, inp, args.cpu_budget, hd)
         line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"first {rows} of {cfg.B} batch rows of {cfg.name}, {dt:.1f} s"}
     print(json.dumps(line), flush=True)
