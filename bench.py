@@ -28,6 +28,10 @@ sys.path.insert(0, str(ROOT))
 
 from paper_2405_19715_b200 import workloads as wl  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one verify/correct call (stats + draw launches), from the ncu
+# captures summarised in profiles/verify_stream_stats_cfg4_B32.md, scaled by units to the full workload.
+NCU_TRAFFIC_BYTES = {"cfg4": 2.329e9}
+
 METRIC = "verified candidate tokens/s"
 UNIT = "tokens/s"
 
@@ -118,6 +122,16 @@ def sum_over_ranks(x: float, world: int, device) -> float:
     return float(t.item())
 
 
+def shard_config(cfg: wl.Workload, rank: int) -> wl.Workload:
+    """Rank r owns its own batch rows (weak scaling): same shapes, a row stream of its own."""
+    return cfg.scaled(seed=cfg.seed + rank)
+
+
+def aggregate(elapsed_ms: float, tokens: float, world: int, device):
+    """Whole-job numbers: the slowest rank's time and the tokens all ranks verified."""
+    return max_over_ranks(elapsed_ms, world, device), sum_over_ranks(tokens, world, device)
+
+
 def barrier(world: int):
     if world > 1:
         import torch.distributed as dist
@@ -202,7 +216,7 @@ def run_ours(args, cfg):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
-    cfg = cfg.scaled(seed=cfg.seed + rank)          # each rank owns its own batch rows
+    cfg = shard_config(cfg, rank)
     inp = wl.make_verify_inputs(cfg)
     lens_np = inp["cand_len"]
     es = 2 if cfg.dtype == "bf16" else 4
@@ -261,12 +275,11 @@ def run_ours(args, cfg):
     torch.cuda.synchronize()
     barrier(world)
     launches = ctx.launch_count() - launches0
-    elapsed_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    elapsed_ms, tokens_step = aggregate(e0.elapsed_time(e1), float(lens_np.sum()), world, dev)
     clocks = sampler.stop() if rank == 0 else None
     verify_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
     head_ms = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
     stop_ms = float(np.mean([e[3].elapsed_time(e[0]) for e in evs]))
-    tokens_step = sum_over_ranks(float(lens_np.sum()), world, dev)
     ms_per_step = elapsed_ms / args.steps
     value = tokens_step / (ms_per_step * 1e-3)
 
@@ -320,7 +333,7 @@ def run_ours(args, cfg):
         "roofline": {"kernel": "verify/correct", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
                      "frac_of_nominal_8TBs": achieved / 8000.0, "algorithmic_bytes": alg, "kernel_ms": verify_ms,
-                     "traffic": None},
+                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name) if args.kernel == 0 else None},
         "parts_ms": {"head": head_ms, "stop": stop_ms, "verify": verify_ms},
         "roofline_head": {"kernel": "acceptance head (2 x [M,4096]x[4096,4096] bf16 GEMM)", "bound": "tensor",
                           "achieved": head_flops / (head_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
