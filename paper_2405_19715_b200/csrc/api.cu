@@ -81,7 +81,7 @@ int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_
         e = cudaMalloc(&ctx->act[0], act);
         if (e == cudaSuccess) e = cudaMalloc(&ctx->act[1], act);
         if (e == cudaSuccess)
-            e = cudaMalloc(&ctx->head_partial, (size_t)max_B * max_K * ((max_d + 127) / 128) * sizeof(float));
+            e = cudaMalloc(&ctx->head_partial, (size_t)max_B * max_K * ((max_d + 63) / 64) * sizeof(float));
     }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {

@@ -4,8 +4,8 @@
 // Each residual block is one GEMM  Z[M, d] = X[M, d] * W^T  (W stored [out, in], so both operands
 // are K-major) on the 5th-generation tensor cores: operand tiles arrive in shared memory by TMA
 // (128-byte swizzle), one thread issues tcgen05.mma with the fp32 accumulator in tensor memory,
-// and four epilogue warps read the accumulator back with tcgen05.ld and apply bias, SiLU and
-// the residual.  The last block does not store x_D: its epilogue multiplies by w_out and leaves
+// and eight epilogue warps read the (double-buffered) accumulator back with tcgen05.ld and apply
+// bias, SiLU and the residual while the next tile's MMAs run.  The last block does not store x_D: its epilogue multiplies by w_out and leaves
 // one partial dot product per (row, column tile); a small kernel adds them and applies the
 // sigmoid.  D = 0 is a plain row-times-vector kernel.
 #include <cuda.h>
@@ -21,7 +21,8 @@ namespace {
 constexpr int BM = 128;                  // rows of X per CTA (= UMMA M)
 constexpr int BK = 64;                   // bf16 elements per k-block: one 128-byte swizzle row
 constexpr int UMMA_K = 16;
-constexpr int HEAD_THREADS = 192;        // warp 0 TMA, warp 1 MMA + tensor-memory owner, warps 2..5 epilogue
+constexpr int EPI_WARPS = 8;             // two per 32-lane quarter of tensor memory, each taking half the columns
+constexpr int HEAD_THREADS = (2 + EPI_WARPS) * 32;   // warp 0 TMA, warp 1 MMA + tensor-memory owner, then epilogue
 constexpr uint32_t WAIT_POLLS = 1u << 24;
 
 template <int BN> struct Cfg {
@@ -35,6 +36,9 @@ template <int BN> struct Cfg {
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
@@ -105,11 +109,15 @@ struct BlockParams {
     const __nv_bfloat16* bias;   // [d] or null
     __nv_bfloat16* Y;            // [M, d] output, null for the last block
     const __nv_bfloat16* w_out;  // [d], last block only
-    float* partial;              // [M, d / BN], last block only
+    float* partial;              // [M, 2 * d / BN], last block only
     int M, d;
+    int sm_count;
     uint32_t* status;
 };
 
+// Persistent: CTA c works on tiles c, c + grid, ... (column tile fastest).  The accumulator is
+// double-buffered in tensor memory (2 x BN columns), so the epilogue of one tile runs while the
+// MMAs of the next are issued.
 template <int BN>
 __global__ void __launch_bounds__(HEAD_THREADS, 1)
 head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
@@ -119,25 +127,29 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
     unsigned char* aligned = smem_raw + (base - smem_u32(smem_raw));
     unsigned long long* bars = reinterpret_cast<unsigned long long*>(aligned + C::STAGES * C::STAGE_BYTES);
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * C::STAGES, tfull = empty0 + 8 * C::STAGES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 1);
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * C::STAGES, tfull0 = empty0 + 8 * C::STAGES,
+                   tempty0 = tfull0 + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int nkb = P.d / BK;
+    const int ntn = P.d / BN, ntiles = ntn * ((P.M + BM - 1) / BM);
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 1);
         }
-        mbar_init(tfull, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull0 + 8 * b, 1);
+            mbar_init(tempty0 + 8 * b, EPI_WARPS);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {                      // this warp owns the tensor-memory allocation
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)BN) : "memory");
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)(2 * BN)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -149,79 +161,104 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
-            for (int kb = 0; kb < nkb; ++kb) {
-                mbar_wait(empty0 + 8 * stage, phase ^ 1u, P.status);
-                const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
-                mbar_expect_tx(full0 + 8 * stage, C::STAGE_BYTES);
-                tma_load_2d(a, &mapX, kb * BK, m0, full0 + 8 * stage);
-                tma_load_2d(b, &mapW, kb * BK, n0, full0 + 8 * stage);
-                if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+            for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
+                const int m0 = (t / ntn) * BM, n0 = (t % ntn) * BN;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    mbar_wait(empty0 + 8 * stage, phase ^ 1u, P.status);
+                    const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
+                    mbar_expect_tx(full0 + 8 * stage, C::STAGE_BYTES);
+                    tma_load_2d(a, &mapX, kb * BK, m0, full0 + 8 * stage);
+                    tma_load_2d(b, &mapW, kb * BK, n0, full0 + 8 * stage);
+                    if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+                }
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc(BN);
-            uint32_t stage = 0, phase = 0;
-            for (int kb = 0; kb < nkb; ++kb) {
-                mbar_wait(full0 + 8 * stage, phase, P.status);
+            uint32_t stage = 0, phase = 0, it = 0;
+            for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
+                const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
+                mbar_wait(tempty0 + 8 * buf, use ^ 1u, P.status);      // epilogue has drained this accumulator
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
+                const uint32_t acc = tmem + buf * BN;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    mbar_wait(full0 + 8 * stage, phase, P.status);
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
 #pragma unroll
-                for (int k = 0; k < BK / UMMA_K; ++k)
-                    umma_bf16(tmem, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), idesc,
-                              (kb | k) != 0 ? 1u : 0u);
-                umma_commit(empty0 + 8 * stage);          // stage reusable once these MMAs have read it
-                if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        umma_bf16(acc, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), idesc,
+                                  (kb | k) != 0 ? 1u : 0u);
+                    umma_commit(empty0 + 8 * stage);          // stage reusable once these MMAs have read it
+                    if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+                }
+                umma_commit(tfull0 + 8 * buf);                // accumulator complete
             }
-            umma_commit(tfull);                            // accumulator complete
         }
     } else {
         // ---------------------------------------------------------------- epilogue warps
         const int q = warp & 3;                            // tensor-memory lane quarter this warp may read
-        const int m = m0 + q * 32 + lane;
-        const bool row_ok = m < P.M;
-        mbar_wait(tfull, 0, P.status);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint4* xrow = reinterpret_cast<const uint4*>(P.X + (size_t)(row_ok ? m : 0) * P.d + n0);
-        float dot = 0.f;
+        const int half = (warp - 2) >> 2;                  // which half of the tile's columns
+        constexpr int CH = BN / 32 / 2;                    // 32-column chunks per warp
+        uint32_t it = 0;
+        for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
+            const int m0 = (t / ntn) * BM, n0 = (t % ntn) * BN;
+            const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
+            const int m = m0 + q * 32 + lane;
+            const bool row_ok = m < P.M;
+            const uint4* xrow = reinterpret_cast<const uint4*>(P.X + (size_t)(row_ok ? m : 0) * P.d + n0);
+            uint4 xv[4], xn[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) xn[j] = row_ok ? __ldg(xrow + (half * CH) * 4 + j) : make_uint4(0, 0, 0, 0);
+            mbar_wait(tfull0 + 8 * buf, use, P.status);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            float dot = 0.f;
 #pragma unroll 1
-        for (int c = 0; c < BN / 32; ++c) {
-            float acc[32];
-            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), acc);
-            uint4 xv[4], bv[4], wv[4];
+            for (int cc = 0; cc < CH; ++cc) {
+                const int c = half * CH + cc;
+                float acc[32];
+                tmem_ld32(tmem + buf * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), acc);
+                uint4 bv[4], wv[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                xv[j] = row_ok ? __ldg(xrow + c * 4 + j) : make_uint4(0, 0, 0, 0);
-                bv[j] = P.bias ? __ldg(reinterpret_cast<const uint4*>(P.bias + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
-                wv[j] = P.w_out ? __ldg(reinterpret_cast<const uint4*>(P.w_out + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
-            }
-            const uint32_t* xw = reinterpret_cast<const uint32_t*>(xv);
-            const uint32_t* bw = reinterpret_cast<const uint32_t*>(bv);
-            const uint32_t* ww = reinterpret_cast<const uint32_t*>(wv);
-            uint32_t out[16];
+                for (int j = 0; j < 4; ++j) {
+                    xv[j] = xn[j];
+                    if (cc + 1 < CH) xn[j] = row_ok ? __ldg(xrow + (c + 1) * 4 + j) : make_uint4(0, 0, 0, 0);
+                    bv[j] = P.bias ? __ldg(reinterpret_cast<const uint4*>(P.bias + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
+                    wv[j] = P.w_out ? __ldg(reinterpret_cast<const uint4*>(P.w_out + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
+                }
+                const uint32_t* xw = reinterpret_cast<const uint32_t*>(xv);
+                const uint32_t* bw = reinterpret_cast<const uint32_t*>(bv);
+                const uint32_t* ww = reinterpret_cast<const uint32_t*>(wv);
+                uint32_t out[16];
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const float y0 = bf16lo(xw[j]) + silu(acc[2 * j] + bf16lo(bw[j]));
-                const float y1 = bf16hi(xw[j]) + silu(acc[2 * j + 1] + bf16hi(bw[j]));
-                dot = fmaf(y0, bf16lo(ww[j]), dot);
-                dot = fmaf(y1, bf16hi(ww[j]), dot);
-                const __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
-                out[j] = *reinterpret_cast<const uint32_t*>(&pk);
-            }
-            if (P.Y && row_ok) {
-                uint4* yrow = reinterpret_cast<uint4*>(P.Y + (size_t)m * P.d + n0 + c * 32);
+                for (int j = 0; j < 16; ++j) {
+                    const float y0 = bf16lo(xw[j]) + silu(acc[2 * j] + bf16lo(bw[j]));
+                    const float y1 = bf16hi(xw[j]) + silu(acc[2 * j + 1] + bf16hi(bw[j]));
+                    dot = fmaf(y0, bf16lo(ww[j]), dot);
+                    dot = fmaf(y1, bf16hi(ww[j]), dot);
+                    const __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
+                    out[j] = *reinterpret_cast<const uint32_t*>(&pk);
+                }
+                if (P.Y && row_ok) {
+                    uint4* yrow = reinterpret_cast<uint4*>(P.Y + (size_t)m * P.d + n0 + c * 32);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) yrow[j] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+                    for (int j = 0; j < 4; ++j) yrow[j] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+                }
             }
+            // this warp has read its part of the accumulator: hand the buffer back to the MMA issuer
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty0 + 8 * buf);
+            if (P.partial && row_ok) P.partial[(size_t)m * (2 * ntn) + 2 * (t % ntn) + half] = dot;
         }
-        if (P.partial && row_ok) P.partial[(size_t)m * gridDim.x + blockIdx.x] = dot;
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)(2 * BN)) : "memory");
     }
 }
 
@@ -288,8 +325,8 @@ template <int BN>
 cudaError_t launch_block(const CUtensorMap& mx, const CUtensorMap& mw, const BlockParams& p, cudaStream_t s) {
     cudaError_t e = cudaFuncSetAttribute(head_block_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM);
     if (e != cudaSuccess) return e;
-    dim3 grid(p.d / BN, (p.M + BM - 1) / BM);
-    head_block_kernel<BN><<<grid, HEAD_THREADS, Cfg<BN>::SMEM, s>>>(mx, mw, p);
+    const int ntiles = (p.d / BN) * ((p.M + BM - 1) / BM);
+    head_block_kernel<BN><<<ntiles < p.sm_count ? ntiles : p.sm_count, HEAD_THREADS, Cfg<BN>::SMEM, s>>>(mx, mw, p);
     return cudaGetLastError();
 }
 
@@ -342,13 +379,14 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
         p.partial = last ? ctx->head_partial : nullptr;
         p.M = (int)M;
         p.d = d;
+        p.sm_count = ctx->sm_count;
         p.status = ctx->status;
         cudaError_t e = BN == 256 ? launch_block<256>(mx, mw, p, s) : launch_block<128>(mx, mw, p, s);
         if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
         ctx->launches += 1;
         x = p.Y;
     }
-    head_finish_kernel<<<(int)((M + 127) / 128), 128, 0, s>>>(ctx->head_partial, (int)M, d / BN, head->b_out, accept_prob);
+    head_finish_kernel<<<(int)((M + 127) / 128), 128, 0, s>>>(ctx->head_partial, (int)M, 2 * d / BN, head->b_out, accept_prob);
     ctx->launches += 1;
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? SPECDEC_OK : fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));

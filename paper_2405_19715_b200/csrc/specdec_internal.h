@@ -26,7 +26,7 @@ struct specdec_ctx {
     size_t stage_bytes = 0;
     // acceptance-head activations (device, bf16) and split-N partial logits
     void* act[2] = {nullptr, nullptr};   // [max_B*max_K, max_d] each
-    float* head_partial = nullptr;       // [max_B*max_K, max_d/128]
+    float* head_partial = nullptr;       // [max_B*max_K, max_d/64]
     char err[256] = "no error";
 };
 
