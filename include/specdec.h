@@ -55,7 +55,10 @@ typedef enum {
 /* Kernel selection for specdec_verify_correct (flags argument). 0 lets the library pick. */
 #define SPECDEC_VERIFY_AUTO    0u
 #define SPECDEC_VERIFY_DIRECT  1u /* one CTA per (row, position), plain global loads      */
-#define SPECDEC_VERIFY_STREAM  2u /* persistent CTAs fed by bulk async copies (TMA)       */
+#define SPECDEC_VERIFY_STREAM  2u /* persistent CTAs fed by bulk async copies (TMA): one launch for the
+                                    statistics and accept tests, a second for the draws           */
+#define SPECDEC_VERIFY_FUSED   3u /* the same pipeline in one launch: CTAs that run out of units
+                                    stream the draws of rows that are already resolved             */
 
 /*
  * Create a context on `device` able to serve calls with B <= max_B and K <= max_K.

@@ -40,7 +40,7 @@ int check_verify_args(specdec_ctx* ctx, const void* target, const void* draft, i
     if (dtype != SPECDEC_F32 && dtype != SPECDEC_BF16) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown dtype %d", dtype);
     if (B < 1 || K < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "verify_correct: B, K, V must be >= 1 (got %d, %d, %d)", B, K, V);
     if (!(T > 0.f) || !std::isfinite(T)) return fail(ctx, SPECDEC_EINVAL, "verify_correct: temperature must be positive and finite");
-    if (flags > SPECDEC_VERIFY_STREAM) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown flags %u", flags);
+    if (flags > SPECDEC_VERIFY_FUSED) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown flags %u", flags);
     if (B > ctx->max_B || K > ctx->max_K)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: B=%d K=%d exceed the context (max_B=%d max_K=%d)", B, K, ctx->max_B, ctx->max_K);
     if (V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: V=%d above 2^22", V);
@@ -71,8 +71,11 @@ int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_
     if (e == cudaSuccess) e = cudaMalloc(&ctx->status, sizeof(uint32_t));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->norms, ndraw * sizeof(float4));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->tasks, (size_t)max_B * sizeof(int2));
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->task_ctl, 2 * sizeof(int32_t));
-    if (e == cudaSuccess) e = cudaMemset(ctx->task_ctl, 0, 2 * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->task_ctl, 8 * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->task_ctl, 0, 8 * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->task_rec, 2 * (size_t)max_B * sizeof(float4));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->task_ready, (size_t)max_B * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemset(ctx->task_ready, 0, (size_t)max_B * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->flags, 0, nflag * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->arrive, 0, (size_t)max_B * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
@@ -103,6 +106,8 @@ int specdec_destroy(specdec_ctx* ctx) {
     cudaFree(ctx->norms);
     cudaFree(ctx->tasks);
     cudaFree(ctx->task_ctl);
+    cudaFree(ctx->task_rec);
+    cudaFree(ctx->task_ready);
     cudaFree(ctx->stage);
     cudaFree(ctx->act[0]);
     cudaFree(ctx->act[1]);
@@ -140,6 +145,7 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     ctx->epoch = (ctx->epoch + 1) & 0x3fffffffu;
     if (ctx->epoch == 0) {   // wrapped: forget every stale flag before reusing epoch numbers
+        CU(ctx, cudaMemsetAsync(ctx->task_ready, 0, (size_t)ctx->max_B * sizeof(int32_t), s));
         CU(ctx, cudaMemsetAsync(ctx->flags, 0, (size_t)ctx->max_B * ctx->max_K * sizeof(int32_t), s));
         ctx->epoch = 1;
     }
@@ -166,22 +172,19 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
     p.norms = ctx->norms;
     p.tasks = ctx->tasks;
     p.task_ctl = ctx->task_ctl;
+    p.task_rec = ctx->task_rec;
+    p.task_ready = ctx->task_ready;
     p.epoch = ctx->epoch;
 
     const bool stream_ok = verify_stream_supported(p, dtype);
-    bool use_stream;
-    if (flags == SPECDEC_VERIFY_STREAM) {
-        if (!stream_ok)
-            return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: streaming kernel needs 16-byte aligned rows (V=%d)", V);
-        use_stream = true;
-    } else if (flags == SPECDEC_VERIFY_DIRECT) {
-        use_stream = false;
-    } else {
-        use_stream = stream_ok;
-    }
+    uint32_t kind = flags;
+    if (kind == SPECDEC_VERIFY_AUTO) kind = stream_ok ? SPECDEC_VERIFY_FUSED : SPECDEC_VERIFY_DIRECT;
+    if (kind != SPECDEC_VERIFY_DIRECT && !stream_ok)
+        return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: streaming kernels need 16-byte aligned rows (V=%d)", V);
     int n_launch = 0;
-    cudaError_t e = use_stream ? launch_verify_stream(p, dtype, ctx->sm_count, s, &n_launch)
-                               : launch_verify_direct(p, dtype, s, &n_launch);
+    cudaError_t e = kind == SPECDEC_VERIFY_FUSED    ? launch_verify_fused(p, dtype, ctx->sm_count, s, &n_launch)
+                    : kind == SPECDEC_VERIFY_STREAM ? launch_verify_stream(p, dtype, ctx->sm_count, s, &n_launch)
+                                                    : launch_verify_direct(p, dtype, s, &n_launch);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "verify_correct launch");
     ctx->launches += n_launch;
     return SPECDEC_OK;

@@ -18,7 +18,9 @@ struct specdec_ctx {
     uint32_t* status = nullptr;   // sticky SPECDEC_DATA_* bits
     float4* norms = nullptr;      // [max_B * (max_K+1)]  log2 normalisers {hi_p, lo_p, hi_q, lo_q} per position
     int2* tasks = nullptr;        // [max_B]              rows whose y' is still to be drawn: {b, n}
-    int32_t* task_ctl = nullptr;  // [2]                  {number of tasks, CTAs of the draw kernel that finished}
+    int32_t* task_ctl = nullptr;  // [8]                  two-launch path: {tasks, finished CTAs}; fused path: {-, -, tail, head, finished}
+    float4* task_rec = nullptr;   // [2 * max_B]          fused path: per resolved row {b, n, mode, u} and its normalisers
+    int32_t* task_ready = nullptr;// [max_B]              fused path: epoch stamp once record t is complete
     uint32_t epoch = 0;
     uint64_t launches = 0;
     // staging for the host-buffer entry point (device), grown on demand
@@ -51,6 +53,8 @@ struct VerifyParams {
     float4* norms;
     int2* tasks;
     int32_t* task_ctl;
+    float4* task_rec;
+    int32_t* task_ready;
     uint32_t epoch;
 };
 
@@ -58,6 +62,8 @@ struct VerifyParams {
 cudaError_t launch_verify_direct(const VerifyParams& p, specdec_dtype dtype, cudaStream_t s, int* n_launch);
 cudaError_t launch_verify_stream(const VerifyParams& p, specdec_dtype dtype, int sm_count, cudaStream_t s,
                                  int* n_launch);
+cudaError_t launch_verify_fused(const VerifyParams& p, specdec_dtype dtype, int sm_count, cudaStream_t s,
+                                int* n_launch);
 bool verify_stream_supported(const VerifyParams& p, specdec_dtype dtype);
 cudaError_t launch_stop(const float* accept_prob, const int32_t* lens, float h, int B, int K,
                         int32_t* stop_pos, cudaStream_t s);

@@ -553,6 +553,354 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) verify_stream_draw_kernel(c
     }
 }
 
+// =============================================================================================
+// Fused kernel: the same pipeline in one launch.  Phase 1 is the statistics pass above.  Every row
+// of the batch ends in exactly one record in a global queue -- {b, n, mode, u, normalisers},
+// written by the epilogue warp that resolves the row (mode 0 for rows that draw nothing: bad
+// length or bad token) and stamped ready with the call's epoch.  When a CTA's producer has
+// streamed its last unit it turns to the queue: it claims record t = head++, waits (bounded) for
+// its stamp, and streams that row pair through the same ring as a draw unit, described to the
+// worker and epilogue warps by a small descriptor ring in shared memory; t >= B ends the CTA.
+// Draws are therefore spread over all CTAs dynamically, overlap the tail of the statistics pass,
+// and find their rows in L2 whenever the batch fits there.  CTAs only ever wait for records of
+// rows whose units belong to CTAs of the same launch (grid <= SM count, one CTA per SM).
+constexpr int DQ = 8;                           // draw descriptors in flight inside a CTA
+constexpr int QD = 2;                           // slab-sum buffers between workers and the draw epilogue
+constexpr uint32_t RECORD_POLLS = 1u << 22;     // bound on the wait for a queue record
+
+struct DrawDesc {
+    int kind;                                   // 0 end of stream, 1 residual draw, 2 draw from the target row
+    int b, n;
+    float u01;
+    Norm np, nq;
+};
+struct FusedShared {
+    StreamShared st;
+    unsigned long long dslot_full[QD];
+    unsigned long long dslot_empty[QD];
+    DrawDesc desc[DQ];
+};
+
+// One queue record for row b (called by one lane).
+__device__ __forceinline__ void push_record(const VerifyParams& P, int b, int n, int mode) {
+    float4 nv = make_float4(0.f, 0.f, 0.f, 0.f);
+    float u01 = 0.f;
+    if (mode) {
+        nv = __ldcg(&P.norms[(size_t)b * (P.K + 1) + n]);
+        u01 = P.uniforms[(size_t)b * (P.K + 1) + P.K];
+    }
+    const int t = atomicAdd(&P.task_ctl[2], 1);
+    P.task_rec[2 * t] = make_float4(__int_as_float(b), __int_as_float(n), __int_as_float(mode), u01);
+    P.task_rec[2 * t + 1] = nv;
+    __threadfence();
+    st_release(&P.task_ready[t], (int)P.epoch);
+}
+
+// next_unit for the fused kernel's reporting warp: a row with a bad length also gets its record.
+__device__ __forceinline__ bool next_unit_fused(const VerifyParams& P, const int* cand_L, int& k, int ncand, Unit& out,
+                                                bool report) {
+    for (; k < ncand; ++k) {
+        const int u = blockIdx.x + k * gridDim.x;
+        const int i = u / P.B, b = u - i * P.B;
+        const int L = k < MAX_CAND ? cand_L[k] : (P.lens ? P.lens[b] : P.K);
+        if (L < 0 || L > P.K) {
+            if (report && i == 0) {
+                atomicOr(P.status, SPECDEC_DATA_BAD_LENGTH);
+                P.n_acc[b] = -1;
+                P.next[b] = -1;
+                if (P.rmass) P.rmass[b] = 0.f;
+                push_record(P, b, 0, 0);
+            }
+            continue;
+        }
+        if (i > L) continue;
+        out.b = b; out.i = i; out.L = L; out.bonus = (i == L);
+        return true;
+    }
+    return false;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(STREAM_THREADS, 1) verify_fused_kernel(const VerifyParams P) {
+    constexpr int N = Elem<T>::EPV;
+    constexpr int NP = N / 2;
+    extern __shared__ __align__(1024) unsigned char smem[];
+    FusedShared& fs = *reinterpret_cast<FusedShared*>(smem + RING_BYTES);
+    StreamShared& ss = fs.st;
+    const int nvec_row = (P.V + N - 1) / N;
+    const int nslab = (nvec_row + 31) / 32;
+    float* slab_base = reinterpret_cast<float*>(smem + RING_BYTES + sizeof(FusedShared));   // [QD][nslab]
+    const uint32_t ring = smem_u32(smem);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    stream_init(ss, tid);
+    if (tid == 0) {
+        for (int s = 0; s < QD; ++s) {
+            mbar_init(smem_u32(&fs.dslot_full[s]), NS);
+            mbar_init(smem_u32(&fs.dslot_empty[s]), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    const int total = (P.K + 1) * P.B;
+    const int ncand = (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    for (int k = tid; k < min(ncand, MAX_CAND); k += STREAM_THREADS) {
+        const int u = blockIdx.x + k * gridDim.x;
+        ss.cand_L[k] = P.lens ? P.lens[u % P.B] : P.K;
+    }
+    __syncthreads();
+
+    const uint32_t row_bytes = (uint32_t)P.V * sizeof(T);
+    const int ntiles = (row_bytes + TILE_BYTES - 1) / TILE_BYTES;
+    int k = 0;
+    Unit un;
+
+    if (warp == NS) {
+        // ================================================================== producer
+        if (lane != 0) return;
+        const unsigned char* tbase = static_cast<const unsigned char*>(P.target);
+        const unsigned char* dbase = static_cast<const unsigned char*>(P.draft);
+        uint32_t stage = 0, phase = 0;
+        while (next_unit(P, ss.cand_L, k, ncand, un, false)) {
+            produce_unit(ss, ring, tbase + ((size_t)un.b * (P.K + 1) + un.i) * row_bytes,
+                         dbase + ((size_t)un.b * P.K + un.i) * row_bytes, un.bonus, row_bytes, ntiles, stage, phase,
+                         P.status);
+            ++k;
+        }
+        // ---- phase 2: draws from the global queue
+        uint32_t seq2 = 0;
+        for (;;) {
+            const int t = atomicAdd(&P.task_ctl[3], 1);
+            if (t >= P.B) break;
+            bool ok = false;
+            for (uint32_t it = 0; it < RECORD_POLLS && !(ok = (ld_acquire(&P.task_ready[t]) == (int)P.epoch)); ++it)
+                __nanosleep(200);
+            if (!ok) { atomicOr(P.status, SPECDEC_DATA_WAIT_LIMIT); continue; }
+            const float4 r0 = __ldcg(&P.task_rec[2 * t]), r1 = __ldcg(&P.task_rec[2 * t + 1]);
+            const int mode = __float_as_int(r0.z);
+            if (mode == 0) continue;
+            const int b = __float_as_int(r0.x), n = __float_as_int(r0.y);
+            // the descriptor must be in place before the unit's first tile can complete
+            mbar_wait(smem_u32(&ss.empty[stage]), phase ^ 1u, P.status);
+            DrawDesc& d = fs.desc[seq2 % DQ];
+            d.kind = mode; d.b = b; d.n = n; d.u01 = r0.w;
+            d.np = Norm{r1.x, r1.y}; d.nq = Norm{r1.z, r1.w};
+            produce_unit(ss, ring, tbase + ((size_t)b * (P.K + 1) + n) * row_bytes,
+                         dbase + ((size_t)b * P.K + n) * row_bytes, mode == 2, row_bytes, ntiles, stage, phase, P.status);
+            ++seq2;
+        }
+        // end marker: an empty stage whose descriptor says "stop"
+        mbar_wait(smem_u32(&ss.empty[stage]), phase ^ 1u, P.status);
+        fs.desc[seq2 % DQ].kind = 0;
+        mbar_arrive(smem_u32(&ss.full[stage]));
+        // the last producer to finish empties the queue counters for the next call
+        __threadfence();
+        if (atomicAdd(&P.task_ctl[4], 1) == (int)gridDim.x - 1) {
+            P.task_ctl[2] = 0;
+            P.task_ctl[3] = 0;
+            P.task_ctl[4] = 0;
+        }
+        return;
+    }
+
+    if (warp < NS) {
+        // ================================================================== worker warps
+        uint32_t stage = 0, phase = 0, seq = 0;
+        while (next_unit(P, ss.cand_L, k, ncand, un, false)) {
+            Acc2 ap = acc2_init(), aq = acc2_init();
+            for (int t = 0; t < ntiles; ++t) {
+                const uint32_t bytes = min((uint32_t)TILE_BYTES, row_bytes - (uint32_t)t * TILE_BYTES);
+                const int nvec = bytes >> 4;
+                const uint32_t base = ring + stage * (2 * TILE_BYTES);
+                mbar_wait_warp(smem_u32(&ss.full[stage]), phase, P.status, lane);
+                uint4 rt[ITERS], rd[ITERS];
+                float mt = -INFINITY, md = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < ITERS; ++j) {
+                    const int v = tid + j * NST;
+                    const uint32_t ninf = neg_inf_word(T());
+                    rt[j] = rd[j] = make_uint4(ninf, ninf, ninf, ninf);
+                    if (v < nvec) {
+                        rt[j] = lds128(base + v * 16);
+                        if (!un.bonus) rd[j] = lds128(base + TILE_BYTES + v * 16);
+                    }
+                    mt = fmaxf(mt, vec_max(rt[j], T()));
+                    md = fmaxf(md, vec_max(rd[j], T()));
+                }
+                acc2_reference(ap, mt, P.c);
+                if (!un.bonus) acc2_reference(aq, md, P.c);
+                const f2 c2 = pack2(P.c, P.c);
+                const f2 np2 = pack2(-ap.rs, -ap.rs), nq2 = pack2(-aq.rs, -aq.rs);
+#pragma unroll
+                for (int j = 0; j < ITERS; ++j) {
+                    f2 xt[NP], xd[NP];
+                    to_pairs(rt[j], xt, T());
+                    acc2_add<NP>(ap, xt, c2, np2);
+                    if (!un.bonus) {
+                        to_pairs(rd[j], xd, T());
+                        acc2_add<NP>(aq, xd, c2, nq2);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ss.empty[stage]));
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            Acc fp = acc2_fold(ap), fq = acc2_fold(aq);      // rs is warp-uniform: add the lanes
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                fp.s += __shfl_xor_sync(0xffffffffu, fp.s, o);
+                fq.s += __shfl_xor_sync(0xffffffffu, fq.s, o);
+            }
+            const uint32_t slot = seq % QSLOTS, use = seq / QSLOTS;
+            if (lane == 0) {
+                if (use > 0) mbar_wait(smem_u32(&ss.slot_empty[slot]), (use - 1) & 1u, P.status);
+                ss.slots[slot][warp] = make_float4(fp.rs, fp.s, fq.rs, fq.s);
+                mbar_arrive(smem_u32(&ss.slot_full[slot]));
+            }
+            ++seq;
+            ++k;
+        }
+        // ---- phase 2: draw units, described by the producer's descriptors
+        for (uint32_t seq2 = 0;; ++seq2) {
+            mbar_wait_warp(smem_u32(&ss.full[stage]), phase, P.status, lane);     // first tile (or the end marker)
+            const DrawDesc d = fs.desc[seq2 % DQ];
+            const uint32_t slot = seq2 % QD, use = seq2 / QD;
+            if (use > 0) mbar_wait_warp(smem_u32(&fs.dslot_empty[slot]), (use - 1) & 1u, P.status, lane);
+            if (d.kind == 0) {                     // pass the end marker on to the draw epilogue
+                if (lane == 0) mbar_arrive(smem_u32(&fs.dslot_full[slot]));
+                break;
+            }
+            float* slab_sum = slab_base + (size_t)slot * nslab;
+            for (int tl = 0; tl < ntiles; ++tl) {
+                const uint32_t bytes = min((uint32_t)TILE_BYTES, row_bytes - (uint32_t)tl * TILE_BYTES);
+                const int nvec = bytes >> 4;
+                const uint32_t base = ring + stage * (2 * TILE_BYTES);
+                if (tl > 0) mbar_wait_warp(smem_u32(&ss.full[stage]), phase, P.status, lane);
+#pragma unroll
+                for (int j = 0; j < ITERS; ++j) {
+                    const int v = tid + j * NST;         // warp-aligned: one slab per warp and j
+                    float ls = 0.f;
+                    if (v < nvec) {
+                        float xt[N], xd[N], w[N];
+                        unpack(lds128(base + v * 16), xt);
+                        if (d.kind == 1) unpack(lds128(base + TILE_BYTES + v * 16), xd);
+                        else {
+#pragma unroll
+                            for (int q = 0; q < N; ++q) xd[q] = 0.f;
+                        }
+                        ls = vec_weights<N>(xt, xd, P.c, d.np, d.nq, d.kind, w);
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, o);
+                    const int slab = tl * (TILE_BYTES / 16 / 32) + j * NS + warp;
+                    if (lane == 0 && slab < nslab) slab_sum[slab] = ls;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ss.empty[stage]));
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (lane == 0) mbar_arrive(smem_u32(&fs.dslot_full[slot]));
+        }
+        return;
+    }
+
+    // ====================================================================== epilogue warps
+    const int e = warp - NS - 1;
+    uint32_t walked = 0;
+    bool have = next_unit_fused(P, ss.cand_L, k, ncand, un, e == 0 && lane == 0);
+    for (;;) {
+        uint32_t seq = 0;
+        if (lane == 0) seq = atomicAdd(&ss.next_seq, 1u);
+        seq = __shfl_sync(0xffffffffu, seq, 0);
+        while (have && walked < seq) {
+            ++k;
+            have = next_unit_fused(P, ss.cand_L, k, ncand, un, e == 0 && lane == 0);
+            ++walked;
+        }
+        if (!have) break;
+        const T* trow = static_cast<const T*>(P.target) + ((size_t)un.b * (P.K + 1) + un.i) * (size_t)P.V;
+        const T* drow = un.bonus ? trow : static_cast<const T*>(P.draft) + ((size_t)un.b * P.K + un.i) * (size_t)P.V;
+        int y_ok = 1;
+        float t_y = 0.f, d_y = 0.f, r = 0.f;
+        if (lane == 0 && !un.bonus) {
+            r = P.uniforms[(size_t)un.b * (P.K + 1) + un.i];
+            const int y = P.tokens[(size_t)un.b * P.K + un.i];
+            y_ok = (y >= 0 && y < P.V);
+            if (y_ok) { t_y = to_float(trow[y]); d_y = to_float(drow[y]); }
+        }
+        const uint32_t slot = seq % QSLOTS, use = seq / QSLOTS;
+        mbar_wait_relaxed(smem_u32(&ss.slot_full[slot]), use & 1u, P.status, lane);
+        Acc a = acc_init(), b = acc_init();
+        if (lane < NS) {
+            const float4 v = ss.slots[slot][lane];
+            a = Acc{v.x, v.y};
+            b = Acc{v.z, v.w};
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ss.slot_empty[slot]));
+        a = warp_merge(a);
+        b = warp_merge(b);
+        if (lane == 0) {
+            const Norm np = make_norm(a), nq = un.bonus ? np : make_norm(b);
+            P.norms[(size_t)un.b * (P.K + 1) + un.i] = make_float4(np.hi, np.lo, nq.hi, nq.lo);
+        }
+        unit_accept(P, un, a, b, t_y, d_y, y_ok, r, lane);
+        if (!row_arrive(P, un, lane)) continue;
+        int n, bad;
+        row_resolve(P, un, lane, n, bad);
+        if (lane == 0) {
+            P.n_acc[un.b] = bad ? -1 : n;
+            if (bad) {
+                P.next[un.b] = -1;
+                if (P.rmass) P.rmass[un.b] = 0.f;
+            }
+            push_record(P, un.b, n, bad ? 0 : (n < un.L ? 1 : 2));
+        }
+    }
+    if (e != 0) return;
+    // ---- phase 2: one epilogue warp picks the tokens of the CTA's draw units
+    for (uint32_t seq2 = 0;; ++seq2) {
+        const uint32_t slot = seq2 % QD, use = seq2 / QD;
+        mbar_wait_relaxed(smem_u32(&fs.dslot_full[slot]), use & 1u, P.status, lane);
+        const DrawDesc d = fs.desc[seq2 % DQ];
+        if (d.kind == 0) break;
+        const int L = P.lens ? P.lens[d.b] : P.K;
+        float* slab_sum = slab_base + (size_t)slot * nslab;
+        const T* trow = static_cast<const T*>(P.target) + ((size_t)d.b * (P.K + 1) + d.n) * (size_t)P.V;
+        const T* drow = d.kind == 2 ? trow : static_cast<const T*>(P.draft) + ((size_t)d.b * P.K + d.n) * (size_t)P.V;
+        double total;
+        int tok = draw_select<T, true>(P, trow, drow, d.kind, d.u01, d.np, d.nq, slab_sum, lane, &total);
+        const double mass = total;
+        if (d.kind == 1 && !(total > 1e-30)) {        // p == q to rounding: draw from p itself (rare)
+            __shared__ UnitShared fallback_sh;
+            if (lane == 0) { fallback_sh.np = d.np; fallback_sh.nq = d.nq; }
+            __syncwarp();
+            unit_draw<T, true>(P, trow, drow, 2, d.u01, fallback_sh, slab_sum, lane, 32, 2);
+            tok = fallback_sh.token;
+        }
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive(smem_u32(&fs.dslot_empty[slot]));
+            P.next[d.b] = tok;
+            if (P.rmass) P.rmass[d.b] = d.n >= L ? 1.f : (float)mass;
+        }
+    }
+}
+
+size_t fused_smem(int V, int elem_size) {
+    const int epv = 16 / elem_size;
+    const int nslab = ((V + epv - 1) / epv + 31) / 32;
+    return (size_t)RING_BYTES + sizeof(FusedShared) + (size_t)QD * nslab * sizeof(float);
+}
+
+template <typename T>
+cudaError_t launch_fused_t(const VerifyParams& p, int sm_count, size_t smem, cudaStream_t s) {
+    cudaError_t e = cudaFuncSetAttribute(verify_fused_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const int total = (p.K + 1) * p.B;
+    verify_fused_kernel<T><<<total < sm_count ? total : sm_count, STREAM_THREADS, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
 size_t stream_smem(int V, int elem_size) {
     const int epv = 16 / elem_size;
     const int nslab = ((V + epv - 1) / epv + 31) / 32;
@@ -579,7 +927,15 @@ bool verify_stream_supported(const VerifyParams& p, specdec_dtype dtype) {
     const int es = dtype == SPECDEC_BF16 ? 2 : 4;
     if (((size_t)p.V * es) % 16 != 0) return false;
     if (reinterpret_cast<uintptr_t>(p.target) % 16 != 0 || reinterpret_cast<uintptr_t>(p.draft) % 16 != 0) return false;
-    return stream_smem(p.V, es) <= 227 * 1024;
+    return stream_smem(p.V, es) <= 227 * 1024 && fused_smem(p.V, es) <= 227 * 1024;
+}
+
+cudaError_t launch_verify_fused(const VerifyParams& p, specdec_dtype dtype, int sm_count, cudaStream_t s,
+                                int* n_launch) {
+    *n_launch = 1;
+    const int es = dtype == SPECDEC_BF16 ? 2 : 4;
+    const size_t smem = fused_smem(p.V, es);
+    return dtype == SPECDEC_BF16 ? launch_fused_t<__nv_bfloat16>(p, sm_count, smem, s) : launch_fused_t<float>(p, sm_count, smem, s);
 }
 
 cudaError_t launch_verify_stream(const VerifyParams& p, specdec_dtype dtype, int sm_count, cudaStream_t s,

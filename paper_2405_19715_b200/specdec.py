@@ -14,7 +14,7 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 OK, EINVAL, EUNSUPPORTED, ECUDA, EDATA = 0, 1, 2, 3, 4
-VERIFY_AUTO, VERIFY_DIRECT, VERIFY_STREAM = 0, 1, 2
+VERIFY_AUTO, VERIFY_DIRECT, VERIFY_STREAM, VERIFY_FUSED = 0, 1, 2, 3
 DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT = 1, 2, 4
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
