@@ -178,7 +178,12 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
 
     const bool stream_ok = verify_stream_supported(p, dtype);
     uint32_t kind = flags;
-    if (kind == SPECDEC_VERIFY_AUTO) kind = stream_ok ? SPECDEC_VERIFY_FUSED : SPECDEC_VERIFY_DIRECT;
+    if (kind == SPECDEC_VERIFY_AUTO) {
+        // The persistent pipeline pays off once the logits clearly exceed what the SMs can pull in a few
+        // round trips; below that the one-CTA-per-unit kernel has the shorter critical path.
+        const double bytes = 2.0 * B * (K + 1.0) * V * (dtype == SPECDEC_BF16 ? 2 : 4);
+        kind = (stream_ok && bytes >= 512e6) ? SPECDEC_VERIFY_FUSED : SPECDEC_VERIFY_DIRECT;
+    }
     if (kind != SPECDEC_VERIFY_DIRECT && !stream_ok)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: streaming kernels need 16-byte aligned rows (V=%d)", V);
     int n_launch = 0;

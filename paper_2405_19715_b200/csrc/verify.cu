@@ -40,38 +40,70 @@ __global__ void __launch_bounds__(DIRECT_THREADS, 2) verify_direct_kernel(const 
     const T* trow = static_cast<const T*>(P.target) + ((size_t)u.b * (P.K + 1) + u.i) * V;
     const T* drow = u.bonus ? trow : static_cast<const T*>(P.draft) + ((size_t)u.b * P.K + u.i) * V;
 
+    // everything the accept test needs besides the sums is requested now and arrives during pass 1
+    int y_ok = 1;
+    float t_y = 0.f, d_y = 0.f, r = 0.f;
+    if (tid == 0 && !u.bonus) {
+        r = P.uniforms[(size_t)u.b * (P.K + 1) + u.i];
+        const int y = P.tokens[(size_t)u.b * P.K + u.i];
+        y_ok = (y >= 0 && y < P.V);
+        if (y_ok) { t_y = to_float(trow[y]); d_y = to_float(drow[y]); }
+    }
+
     // ---- pass 1: softmax statistics of both rows
     const int nvec = (P.V + N - 1) / N;
     Acc ap = acc_init(), aq = acc_init();
-    float xt[N], xd[N], xt2[N], xd2[N];
-    int j = tid;
-    if (!u.bonus) {
-        for (; j + DIRECT_THREADS < nvec; j += 2 * DIRECT_THREADS) {
-            load_vec<T, VEC>(trow, j, P.V, xt);
-            load_vec<T, VEC>(drow, j, P.V, xd);
-            load_vec<T, VEC>(trow, j + DIRECT_THREADS, P.V, xt2);
-            load_vec<T, VEC>(drow, j + DIRECT_THREADS, P.V, xd2);
-            acc_update<N>(ap, xt, P.c);
-            acc_update<N>(aq, xd, P.c);
-            acc_update<N>(ap, xt2, P.c);
-            acc_update<N>(aq, xd2, P.c);
+    if constexpr (VEC) {
+        // four vectors of each row in flight per thread; the reference is moved from the maximum of
+        // the raw inputs, so the exponentials are issued without a data-dependent branch
+        constexpr int U = 4, NP = N / 2;
+        const uint4* tv = reinterpret_cast<const uint4*>(trow);
+        const uint4* dv = reinterpret_cast<const uint4*>(drow);
+        const uint32_t ninf = neg_inf_word(T());
+        Acc2 a2 = acc2_init(), q2 = acc2_init();
+        for (int j0 = tid; j0 < nvec; j0 += U * DIRECT_THREADS) {
+            uint4 rt[U], rd[U];
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                const int j = j0 + k * DIRECT_THREADS;
+                rt[k] = rd[k] = make_uint4(ninf, ninf, ninf, ninf);
+                if (j < nvec) {
+                    rt[k] = __ldcg(tv + j);
+                    if (!u.bonus) rd[k] = __ldcg(dv + j);
+                }
+            }
+            float mt = -INFINITY, md = -INFINITY;
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                mt = fmaxf(mt, vec_max(rt[k], T()));
+                md = fmaxf(md, vec_max(rd[k], T()));
+            }
+            acc2_reference_thread(a2, mt, P.c);
+            if (!u.bonus) acc2_reference_thread(q2, md, P.c);
+            const f2 c2 = pack2(P.c, P.c);
+            const f2 np2 = pack2(-a2.rs, -a2.rs), nq2 = pack2(-q2.rs, -q2.rs);
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                f2 xt[NP], xd[NP];
+                to_pairs(rt[k], xt, T());
+                acc2_add<NP>(a2, xt, c2, np2);
+                if (!u.bonus) {
+                    to_pairs(rd[k], xd, T());
+                    acc2_add<NP>(q2, xd, c2, nq2);
+                }
+            }
         }
-        if (j < nvec) {
-            load_vec<T, VEC>(trow, j, P.V, xt);
-            load_vec<T, VEC>(drow, j, P.V, xd);
-            acc_update<N>(ap, xt, P.c);
-            acc_update<N>(aq, xd, P.c);
-        }
+        ap = acc2_fold(a2);
+        aq = acc2_fold(q2);
     } else {
-        for (; j + DIRECT_THREADS < nvec; j += 2 * DIRECT_THREADS) {
-            load_vec<T, VEC>(trow, j, P.V, xt);
-            load_vec<T, VEC>(trow, j + DIRECT_THREADS, P.V, xt2);
-            acc_update<N>(ap, xt, P.c);
-            acc_update<N>(ap, xt2, P.c);
-        }
-        if (j < nvec) {
+        float xt[N], xd[N];
+        for (int j = tid; j < nvec; j += DIRECT_THREADS) {
             load_vec<T, VEC>(trow, j, P.V, xt);
             acc_update<N>(ap, xt, P.c);
+            if (!u.bonus) {
+                load_vec<T, VEC>(drow, j, P.V, xd);
+                acc_update<N>(aq, xd, P.c);
+            }
         }
     }
     ap = warp_merge(ap);
@@ -83,14 +115,6 @@ __global__ void __launch_bounds__(DIRECT_THREADS, 2) verify_direct_kernel(const 
         Acc a = lane < NW ? sh.wp[lane] : acc_init(), b = lane < NW ? sh.wq[lane] : acc_init();
         a = warp_merge(a);
         b = warp_merge(b);
-        int y = 0, y_ok = 1;
-        float t_y = 0.f, d_y = 0.f, r = 0.f;
-        if (lane == 0 && !u.bonus) {
-            r = P.uniforms[(size_t)u.b * (P.K + 1) + u.i];
-            y = P.tokens[(size_t)u.b * P.K + u.i];
-            y_ok = (y >= 0 && y < P.V);
-            if (y_ok) { t_y = to_float(trow[y]); d_y = to_float(drow[y]); }
-        }
         const int mode = unit_decide(P, u, a, b, t_y, d_y, y_ok, r, lane);
         if (lane == 0) {
             sh.np = make_norm(a);

@@ -120,6 +120,114 @@ __device__ __forceinline__ void acc_update(Acc& a, const float (&x)[N], float c)
     a.s += vs;
 }
 
+// ---- packed fp32x2 arithmetic ------------------------------------------------------------
+using f2 = unsigned long long;
+__device__ __forceinline__ f2 pack2(float a, float b) {
+    f2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f2 v, float& a, float& b) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c) {
+    f2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f2 add2(f2 a, f2 b) {
+    f2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f2 mul2(f2 a, f2 b) {
+    f2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f2 ex2_2(f2 a) {
+    float x, y;
+    unpack2(a, x, y);
+    return pack2(ex2(x), ex2(y));
+}
+
+// Statistics of one row inside a statistics warp: every lane keeps two interleaved partial sums
+// of 2^(x*c - rs) against a reference rs that is the same in all lanes of the warp.  Before a
+// tile's exponentials are issued the warp takes the maximum of the tile's raw logits (packed
+// max, one redux) and moves the reference up if that maximum sits more than 8 binades above it,
+// so the hot loop has no data-dependent branch, exponent arguments of the terms that matter
+// stay small, and nothing can overflow.
+struct Acc2 {
+    float rs;
+    f2 s;
+};
+__device__ __forceinline__ Acc2 acc2_init() { return Acc2{NEG_BIG, pack2(0.f, 0.f)}; }
+__device__ __forceinline__ Acc acc2_fold(const Acc2& a) {
+    float lo, hi;
+    unpack2(a.s, lo, hi);
+    return Acc{a.rs, lo + hi};
+}
+
+__device__ __forceinline__ uint32_t max_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// Largest element of a 16-byte vector as fp32 (NaNs are skipped).
+__device__ __forceinline__ float vec_max(const uint4& r, __nv_bfloat16) {
+    const uint32_t m = max_bf16x2(max_bf16x2(r.x, r.y), max_bf16x2(r.z, r.w));
+    return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xffff0000u));
+}
+__device__ __forceinline__ float vec_max(const uint4& r, float) {
+    return fmaxf(fmaxf(__uint_as_float(r.x), __uint_as_float(r.y)), fmaxf(__uint_as_float(r.z), __uint_as_float(r.w)));
+}
+__device__ __forceinline__ uint32_t neg_inf_word(__nv_bfloat16) { return 0xff80ff80u; }
+__device__ __forceinline__ uint32_t neg_inf_word(float) { return 0xff800000u; }
+
+// Warp-uniform re-reference: m is this lane's maximum raw logit of the coming tile.
+__device__ __forceinline__ void acc2_reference(Acc2& a, float m, float c) {
+    float M;
+    asm("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(M) : "f"(m));
+    const float top = M * c;
+    if (top > a.rs + 8.f && M > -3.0e38f) {          // same decision in every lane
+        const float f = ex2(a.rs - top);
+        a.s = mul2(a.s, pack2(f, f));
+        a.rs = top;
+    }
+}
+
+// The same decision taken by one thread for itself (kernels whose threads keep references of
+// their own).
+__device__ __forceinline__ void acc2_reference_thread(Acc2& a, float m, float c) {
+    const float top = m * c;
+    if (top > a.rs + 8.f && m > -3.0e38f) {
+        const float f = ex2(a.rs - top);
+        a.s = mul2(a.s, pack2(f, f));
+        a.rs = top;
+    }
+}
+
+template <int NP>   // NP packed pairs = 2*NP elements of one 16-byte vector
+__device__ __forceinline__ void acc2_add(Acc2& a, const f2 (&x)[NP], f2 c2, f2 nrs) {
+    f2 e[NP];
+#pragma unroll
+    for (int k = 0; k < NP; ++k) e[k] = ex2_2(fma2(x[k], c2, nrs));
+    if constexpr (NP == 4) a.s = add2(a.s, add2(add2(e[0], e[1]), add2(e[2], e[3])));
+    else a.s = add2(a.s, add2(e[0], e[1]));
+}
+
+__device__ __forceinline__ void to_pairs(const uint4& r, f2 (&x)[2], float) {          // 4 fp32
+    x[0] = pack2(__uint_as_float(r.x), __uint_as_float(r.y));
+    x[1] = pack2(__uint_as_float(r.z), __uint_as_float(r.w));
+}
+__device__ __forceinline__ void to_pairs(const uint4& r, f2 (&x)[4], __nv_bfloat16) {  // 8 bf16, widened exactly
+    x[0] = pack2(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u));
+    x[1] = pack2(__uint_as_float(r.y << 16), __uint_as_float(r.y & 0xffff0000u));
+    x[2] = pack2(__uint_as_float(r.z << 16), __uint_as_float(r.z & 0xffff0000u));
+    x[3] = pack2(__uint_as_float(r.w << 16), __uint_as_float(r.w & 0xffff0000u));
+}
+
+
 __device__ __forceinline__ Acc acc_merge(const Acc& a, const Acc& b) {
     Acc r;
     r.rs = fmaxf(a.rs, b.rs);
