@@ -125,6 +125,25 @@ int specdec_verify_correct(specdec_ctx* ctx,
                            uint32_t flags, void* stream);
 
 /*
+ * Greedy verification (Section 4.1: the deterministic setting in which both models decode
+ * greedily).  The drafted tokens are given; candidate i is kept while it equals the target's
+ * argmax at position i, the first mismatch is replaced by that argmax, and when all cand_len[b]
+ * candidates match, the target's argmax at position cand_len[b] is appended.  Only target rows
+ * 0..cand_len[b] are read.  Ties in a row resolve to the lowest token index.
+ *
+ *   target_logits dev [B, K+1, V], cand_tokens dev [B, K] int32, cand_len dev [B] int32 or NULL
+ *   n_accepted    dev out [B] int32   number of leading candidates equal to the target's argmax
+ *   next_token    dev out [B] int32   target argmax at position n_accepted[b]
+ *   target_argmax dev out [B, K+1] int32 or NULL: argmax of every row that was read, -1 elsewhere
+ * Errors and device-side data checks as for specdec_verify_correct.
+ */
+int specdec_verify_greedy(specdec_ctx* ctx, const void* target_logits, specdec_dtype dtype,
+                          const int32_t* cand_tokens, const int32_t* cand_len,
+                          int B, int K, int V,
+                          int32_t* n_accepted, int32_t* next_token, int32_t* target_argmax,
+                          void* stream);
+
+/*
  * Same operation with HOST input and output buffers: copies the inputs to device staging
  * buffers owned by the context (allocated or grown on first use), runs the kernels, copies
  * n_accepted / next_token (and accept_ratio when not NULL) back and synchronises `stream`
@@ -172,6 +191,16 @@ int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const specdec_head
  */
 int specdec_stop(specdec_ctx* ctx, const float* accept_prob, const int32_t* cand_len,
                  float h, int B, int K, int32_t* stop_pos, void* stream);
+
+/*
+ * One trip of Algorithm 1's drafting loop for B sequences (the online form of specdec_stop):
+ *   p_hat[b] <- p_hat[b] * accept_prob_step[b];   stop[b] = (1 - p_hat[b] > h) ? 1 : 0.
+ * The caller starts a speculation round with p_hat = 1 and calls this after each drafted token
+ * with the head's output for that token (specdec_accept_head with K = 1).
+ *   accept_prob_step dev [B] f32, p_hat dev in/out [B] f32, stop dev out [B] int32
+ */
+int specdec_stop_step(specdec_ctx* ctx, const float* accept_prob_step, float* p_hat, float h, int B,
+                      int32_t* stop, void* stream);
 
 /*
  * Allocation-free variant of specdec_verify_correct.  The paper has no counterpart: this entry

@@ -42,7 +42,7 @@ __all__ = [
     "bf16_bits_to_f64", "logits_to_f64", "softmax_T", "log_sum_exp_T",
     "accept_ratio", "first_rejection", "residual", "inverse_cdf",
     "verify_from_probs", "verify_correct", "sampling_weights",
-    "silu", "sigmoid", "accept_head", "stop_rule", "greedy_verify",
+    "silu", "sigmoid", "accept_head", "stop_rule", "greedy_verify", "greedy_verify_tokens", "stop_step",
 ]
 
 
@@ -223,22 +223,34 @@ def verify_correct(target_logits, draft_logits, cand_tokens, cand_len, uniforms,
     return out
 
 
-def greedy_verify(target_logits, draft_logits, cand_len=None):
-    """Greedy special case (Section 4.1): the draft proposes argmax q_i, a candidate is
-    kept while it equals argmax p_i, the first mismatch is replaced by argmax p_i, and
-    argmax p_{L} is appended when all match.  Ties resolve to the lowest index."""
+def greedy_verify_tokens(target_logits, cand_tokens, cand_len=None):
+    """Greedy special case (Section 4.1) with the drafted tokens given: a candidate is kept while
+    it equals argmax p_i, the first mismatch is replaced by argmax p_i, and argmax p_L is appended
+    when all L candidates match.  Ties resolve to the lowest index.  Returns (n_accepted,
+    next_token, target_argmax [B,K+1] with -1 at rows the method does not look at)."""
     t = logits_to_f64(np.asarray(target_logits))
-    d = logits_to_f64(np.asarray(draft_logits))
     B, K1, _ = t.shape
+    y = np.asarray(cand_tokens).reshape(B, K1 - 1)
     lens = np.full(B, K1 - 1) if cand_len is None else np.asarray(cand_len)
     n_acc, nxt = np.zeros(B, np.int32), np.zeros(B, np.int32)
+    am = np.full((B, K1), -1, np.int32)
     for b in range(B):
-        n = int(lens[b])
-        for i in range(int(lens[b])):
-            if int(np.argmax(d[b, i])) != int(np.argmax(t[b, i])):
+        L = int(lens[b])
+        for i in range(L + 1):
+            am[b, i] = int(np.argmax(t[b, i]))
+        n = L
+        for i in range(L):
+            if int(y[b, i]) != am[b, i]:
                 n = i
                 break
-        n_acc[b], nxt[b] = n, int(np.argmax(t[b, n]))
+        n_acc[b], nxt[b] = n, am[b, n]
+    return n_acc, nxt, am
+
+
+def greedy_verify(target_logits, draft_logits, cand_len=None):
+    """Greedy special case (Section 4.1): the draft proposes argmax q_i; see greedy_verify_tokens."""
+    d = logits_to_f64(np.asarray(draft_logits))
+    n_acc, nxt, _ = greedy_verify_tokens(target_logits, d.argmax(-1), cand_len)
     return n_acc, nxt
 
 
@@ -292,3 +304,12 @@ def stop_rule(accept_prob, h, cand_len=None):
                 break
         out[b] = pos
     return out
+
+
+def stop_step(p_hat, accept_prob_step, h):
+    """One trip of Algorithm 1's drafting loop for a batch: p_hat <- p_hat * sigmoid(f(e)) and the
+    decision 1 - p_hat > h.  p_hat, accept_prob_step: [B] float32 values (used exactly, in float64).
+    Returns (new p_hat [B] float64, stop [B] bool)."""
+    p = np.asarray(p_hat, dtype=np.float64) * np.asarray(accept_prob_step, dtype=np.float32).astype(np.float64)
+    return p, (1.0 - p) > float(np.float32(h))
+

@@ -84,7 +84,7 @@ int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_
         e = cudaMalloc(&ctx->act[0], act);
         if (e == cudaSuccess) e = cudaMalloc(&ctx->act[1], act);
         if (e == cudaSuccess)
-            e = cudaMalloc(&ctx->head_partial, (size_t)max_B * max_K * ((max_d + 63) / 64) * sizeof(float));
+            e = cudaMalloc(&ctx->head_partial, (size_t)max_B * max_K * ((max_d + 31) / 32) * sizeof(float));
     }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -195,6 +195,43 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
     return SPECDEC_OK;
 }
 
+int specdec_verify_greedy(specdec_ctx* ctx, const void* target_logits, specdec_dtype dtype,
+                          const int32_t* cand_tokens, const int32_t* cand_len, int B, int K, int V,
+                          int32_t* n_accepted, int32_t* next_token, int32_t* target_argmax, void* stream) {
+    if (!ctx) return SPECDEC_EINVAL;
+    if (!target_logits || !cand_tokens || !n_accepted || !next_token)
+        return fail(ctx, SPECDEC_EINVAL, "verify_greedy: null pointer argument");
+    if (dtype != SPECDEC_F32 && dtype != SPECDEC_BF16) return fail(ctx, SPECDEC_EINVAL, "verify_greedy: unknown dtype %d", (int)dtype);
+    if (B < 1 || K < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "verify_greedy: B, K, V must be >= 1");
+    if (B > ctx->max_B || K > ctx->max_K)
+        return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_greedy: B=%d K=%d exceed the context (max_B=%d max_K=%d)", B, K, ctx->max_B, ctx->max_K);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    ctx->epoch = (ctx->epoch + 1) & 0x3fffffffu;
+    if (ctx->epoch == 0) {
+        CU(ctx, cudaMemsetAsync(ctx->task_ready, 0, (size_t)ctx->max_B * sizeof(int32_t), s));
+        CU(ctx, cudaMemsetAsync(ctx->flags, 0, (size_t)ctx->max_B * ctx->max_K * sizeof(int32_t), s));
+        ctx->epoch = 1;
+    }
+    VerifyParams p = {};
+    p.target = target_logits;
+    p.tokens = cand_tokens;
+    p.lens = cand_len;
+    p.B = B;
+    p.K = K;
+    p.V = V;
+    p.n_acc = n_accepted;
+    p.next = next_token;
+    p.flags = ctx->flags;
+    p.draws = ctx->draws;
+    p.arrive = ctx->arrive;
+    p.status = ctx->status;
+    p.epoch = ctx->epoch;
+    cudaError_t e = launch_greedy(p, dtype, target_argmax, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "verify_greedy launch");
+    ctx->launches += 1;
+    return SPECDEC_OK;
+}
+
 int specdec_verify_correct_host(specdec_ctx* ctx, const void* target_logits, const void* draft_logits,
                                 specdec_dtype dtype, const int32_t* cand_tokens, const int32_t* cand_len,
                                 const float* uniforms, float temperature, int B, int K, int V,
@@ -252,6 +289,18 @@ int specdec_stop(specdec_ctx* ctx, const float* accept_prob, const int32_t* cand
     if (h != h) return fail(ctx, SPECDEC_EINVAL, "stop: threshold is NaN");
     cudaError_t e = launch_stop(accept_prob, cand_len, h, B, K, stop_pos, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "stop launch");
+    ctx->launches += 1;
+    return SPECDEC_OK;
+}
+
+int specdec_stop_step(specdec_ctx* ctx, const float* accept_prob_step, float* p_hat, float h, int B,
+                      int32_t* stop, void* stream) {
+    if (!ctx) return SPECDEC_EINVAL;
+    if (!accept_prob_step || !p_hat || !stop) return fail(ctx, SPECDEC_EINVAL, "stop_step: null pointer argument");
+    if (B < 1) return fail(ctx, SPECDEC_EINVAL, "stop_step: B must be >= 1");
+    if (h != h) return fail(ctx, SPECDEC_EINVAL, "stop_step: threshold is NaN");
+    cudaError_t e = launch_stop_step(accept_prob_step, p_hat, h, B, stop, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "stop_step launch");
     ctx->launches += 1;
     return SPECDEC_OK;
 }

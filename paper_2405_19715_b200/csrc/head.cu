@@ -26,7 +26,7 @@ constexpr int HEAD_THREADS = (2 + EPI_WARPS) * 32;   // warp 0 TMA, warp 1 MMA +
 constexpr uint32_t WAIT_POLLS = 1u << 24;
 
 template <int BN> struct Cfg {
-    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
@@ -361,7 +361,9 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
         cudaError_t e = cudaGetLastError();
         return e == cudaSuccess ? SPECDEC_OK : fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
     }
-    const int BN = d % 256 == 0 ? 256 : 128;
+    // few rows (the online, one-token-per-call use): narrow column tiles so that the weight stream is
+    // spread over many SMs; otherwise the widest tile the width allows
+    const int BN = M <= 256 ? 64 : (d % 256 == 0 ? 256 : 128);
     for (int k = 0; k < D; ++k) {
         const void* W = head->W[k];
         const void* bias = head->b ? head->b[k] : nullptr;
@@ -381,7 +383,8 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
         p.d = d;
         p.sm_count = ctx->sm_count;
         p.status = ctx->status;
-        cudaError_t e = BN == 256 ? launch_block<256>(mx, mw, p, s) : launch_block<128>(mx, mw, p, s);
+        cudaError_t e = BN == 256 ? launch_block<256>(mx, mw, p, s)
+                        : BN == 128 ? launch_block<128>(mx, mw, p, s) : launch_block<64>(mx, mw, p, s);
         if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
         ctx->launches += 1;
         x = p.Y;

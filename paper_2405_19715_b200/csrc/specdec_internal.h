@@ -28,7 +28,7 @@ struct specdec_ctx {
     size_t stage_bytes = 0;
     // acceptance-head activations (device, bf16) and split-N partial logits
     void* act[2] = {nullptr, nullptr};   // [max_B*max_K, max_d] each
-    float* head_partial = nullptr;       // [max_B*max_K, max_d/64]
+    float* head_partial = nullptr;       // [max_B*max_K, max_d/32]
     char err[256] = "no error";
 };
 
@@ -65,5 +65,8 @@ cudaError_t launch_verify_stream(const VerifyParams& p, specdec_dtype dtype, int
 cudaError_t launch_verify_fused(const VerifyParams& p, specdec_dtype dtype, int sm_count, cudaStream_t s,
                                 int* n_launch);
 bool verify_stream_supported(const VerifyParams& p, specdec_dtype dtype);
+cudaError_t launch_greedy(const VerifyParams& p, specdec_dtype dtype, int32_t* argmax_out, cudaStream_t s);
 cudaError_t launch_stop(const float* accept_prob, const int32_t* lens, float h, int B, int K,
                         int32_t* stop_pos, cudaStream_t s);
+cudaError_t launch_stop_step(const float* accept_prob_step, float* p_hat, float h, int B, int32_t* stop,
+                             cudaStream_t s);

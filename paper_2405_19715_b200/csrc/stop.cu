@@ -20,7 +20,23 @@ __global__ void stop_kernel(const float* __restrict__ a, const int32_t* __restri
     stop_pos[b] = pos;
 }
 
+// One trip of Algorithm 1's loop for every row: p_hat <- p_hat * a; stop iff 1 - p_hat > h.
+__global__ void stop_step_kernel(const float* __restrict__ a, float* __restrict__ p_hat, float h, int B,
+                                 int32_t* __restrict__ stop) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const float p = p_hat[b] * a[b];
+    p_hat[b] = p;
+    stop[b] = (1.f - p > h) ? 1 : 0;
+}
+
 }  // namespace
+
+cudaError_t launch_stop_step(const float* accept_prob_step, float* p_hat, float h, int B, int32_t* stop,
+                             cudaStream_t s) {
+    stop_step_kernel<<<(B + 127) / 128, 128, 0, s>>>(accept_prob_step, p_hat, h, B, stop);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_stop(const float* accept_prob, const int32_t* lens, float h, int B, int K, int32_t* stop_pos,
                         cudaStream_t s) {

@@ -19,7 +19,7 @@ DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT = 1, 2, 4
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
            "specdec_launch_count", "specdec_verify_correct", "specdec_verify_correct_host",
-           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static"]
+           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step"]
 STATIC_MAX_UNITS, STATIC_MAX_V = 16384, 262144
 
 
@@ -58,6 +58,9 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
                                                 C.c_int, C.c_int, ip, ip, fp, C.c_uint32, C.c_void_p]
     lib.specdec_accept_head.argtypes = [C.c_void_p, vp, C.POINTER(_Head), C.c_int, C.c_int, fp, C.c_void_p]
     lib.specdec_stop.argtypes = [C.c_void_p, fp, ip, C.c_float, C.c_int, C.c_int, ip, C.c_void_p]
+    lib.specdec_stop_step.argtypes = [C.c_void_p, fp, fp, C.c_float, C.c_int, ip, C.c_void_p]
+    lib.specdec_verify_greedy.argtypes = [C.c_void_p, vp, C.c_int, ip, ip, C.c_int, C.c_int, C.c_int, ip, ip, ip,
+                                          C.c_void_p]
     lib.specdec_verify_correct_static.argtypes = [vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int, C.c_int, C.c_int,
                                                   ip, ip, C.c_void_p, C.c_void_p, C.c_char_p, C.c_size_t]
     if path is None:
@@ -182,6 +185,34 @@ def specdec_verify_correct_host(ctx: Context, target_logits, draft_logits, cand_
         _ptr(uniforms, torch.float32, False), float(temperature), B, K, V,
         _ptr(n_accepted, torch.int32, False), _ptr(next_token, torch.int32, False),
         _ptr(accept_ratio, torch.float32, False), flags, _stream(stream))
+    ctx._check(rc)
+    return n_accepted, next_token
+
+
+def specdec_stop_step(ctx: Context, accept_prob_step, p_hat, h: float, stop=None, stream=None):
+    """specdec_stop_step of the C ABI: updates p_hat in place, returns stop [B] int32."""
+    B = accept_prob_step.numel()
+    if stop is None:
+        stop = torch.empty(B, dtype=torch.int32, device=p_hat.device)
+    rc = ctx.lib.specdec_stop_step(ctx.handle, _ptr(accept_prob_step, torch.float32), _ptr(p_hat, torch.float32),
+                                   float(h), B, _ptr(stop, torch.int32), _stream(stream))
+    ctx._check(rc)
+    return stop
+
+
+def specdec_verify_greedy(ctx: Context, target_logits, cand_tokens, cand_len=None, n_accepted=None, next_token=None,
+                          target_argmax=None, stream=None):
+    """specdec_verify_greedy of the C ABI.  Returns (n_accepted, next_token) device tensors."""
+    B, K1, V = target_logits.shape
+    dev = target_logits.device
+    if n_accepted is None:
+        n_accepted = torch.empty(B, dtype=torch.int32, device=dev)
+    if next_token is None:
+        next_token = torch.empty(B, dtype=torch.int32, device=dev)
+    rc = ctx.lib.specdec_verify_greedy(ctx.handle, _ptr(target_logits), _logit_dtype(target_logits),
+                                       _ptr(cand_tokens, torch.int32), _ptr(cand_len, torch.int32), B, K1 - 1, V,
+                                       _ptr(n_accepted, torch.int32), _ptr(next_token, torch.int32),
+                                       _ptr(target_argmax, torch.int32), _stream(stream))
     ctx._check(rc)
     return n_accepted, next_token
 

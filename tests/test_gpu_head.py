@@ -35,8 +35,10 @@ def _run_head(ctx, hidden, Ws, bs, w_out, b_out):
 @pytest.mark.parametrize("d", [128, 256, 384, 512])
 @pytest.mark.parametrize("depth", [0, 1, 2, 3])
 @pytest.mark.parametrize("with_bias", [False, True])
-def test_head_small_shapes(d, depth, with_bias):
-    B, K = 7, 23                      # 161 rows: one full 128-row tile and a ragged one
+@pytest.mark.parametrize("rows", [(7, 23), (9, 33)], ids=["161rows", "297rows"])
+def test_head_small_shapes(d, depth, with_bias, rows):
+    B, K = rows                       # 161 rows use the narrow 64-column tiles, 297 rows the 128/256-column ones;
+                                      # both leave a ragged last row tile
     ctx = specdec.Context(B, K, max_d=d)
     hidden, Ws, bs, w_out, b_out = _head_problem(100 + d + depth, B, K, d, depth, with_bias)
     got = _run_head(ctx, hidden, Ws, bs, w_out, b_out)
@@ -98,5 +100,41 @@ def test_config5_head_stop_verify_chain():
     gpu = parity.run_gpu_verify(ctx, inp)
     rep = parity.classify_rows(inp, gpu, dtype="f32")
     print("cfg5 verify", rep)
+    assert ctx.device_status() == 0
+    ctx.close()
+
+
+def test_online_head_and_stop_step_replay_algorithm_1():
+    """Algorithm 1's loop, one drafted token per call: head on [B,1,d] (narrow-tile GEMM), then
+    specdec_stop_step.  Each step is checked against the oracle; the replay must also reproduce the
+    batched head + stop rule."""
+    B, K, d = 96, 6, 512
+    ctx = specdec.Context(B, K, max_d=d)
+    hidden, Ws, bs, w_out, b_out = _head_problem(77, B, K, d, 2, True, std=0.03)
+    batched = _run_head(ctx, hidden, Ws, bs, w_out, b_out)                      # [B, K]
+    tW = [specdec.from_numpy(w) for w in Ws]
+    tb = [specdec.from_numpy(b) for b in bs]
+    tw = specdec.from_numpy(w_out)
+    h = 0.5
+    p_hat = torch.ones(B, dtype=torch.float32, device="cuda")
+    o_hat = np.ones(B)
+    first = np.full(B, K)
+    for j in range(K):
+        step_hidden = np.ascontiguousarray(hidden[:, j:j + 1, :])
+        a = specdec.specdec_accept_head(ctx, specdec.from_numpy(step_hidden), tW, tb, tw, b_out)   # [B, 1]
+        want = orc.accept_head(step_hidden, list(zip(Ws, bs)), w_out, b_out)
+        got = a.cpu().numpy()
+        assert np.max(np.abs(got - want) / want) <= HEAD_RTOL
+        np.testing.assert_allclose(got[:, 0], batched[:, j], rtol=1e-4)
+        stop = specdec.specdec_stop_step(ctx, a.reshape(B), p_hat, h).cpu().numpy()
+        o_hat, o_stop = orc.stop_step(o_hat.astype(np.float32), got[:, 0], h)
+        near = np.abs(1.0 - o_hat - np.float32(h)) < parity.BOUNDARY
+        assert np.array_equal(stop[~near].astype(bool), o_stop[~near])
+        np.testing.assert_allclose(p_hat.cpu().numpy(), o_hat, rtol=1e-6)
+        first = np.where((first == K) & (stop == 1), j, first)
+    pos = specdec.specdec_stop(ctx, torch.from_numpy(batched).cuda(), h).cpu().numpy()
+    rep = parity.classify_stop(batched, h, pos)
+    assert rep["exact"] + rep["boundary"] == B
+    assert (first == pos).mean() > 0.95          # identical except where a product sits on the threshold
     assert ctx.device_status() == 0
     ctx.close()

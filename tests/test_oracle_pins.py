@@ -390,6 +390,22 @@ def test_stop_rule_closed_form_and_monotone():
     assert np.array_equal(out, lens)
 
 
+def test_stop_step_iterated_equals_stop_rule():
+    """Algorithm 1 applies the update one drafted token at a time; iterating it is the batched rule."""
+    rng = np.random.default_rng(17)
+    probs = rng.uniform(0.4, 1.0, size=(40, 12)).astype(np.float32)
+    for h in (0.2, 0.5, 0.8):
+        want = orc.stop_rule(probs, h)
+        p_hat = np.ones(40)
+        first = np.full(40, 12)
+        for j in range(12):
+            p_hat, stop = orc.stop_step(p_hat, probs[:, j], h)
+            first = np.where((first == 12) & stop, j, first)
+        assert np.array_equal(first, want)
+    p, stop = orc.stop_step(np.array([1.0, 0.5]), np.array([0.5, 0.5], np.float32), 0.5)
+    assert p.tolist() == [0.5, 0.25] and stop.tolist() == [False, True]      # strict: 1 - 0.5 > 0.5 is false
+
+
 # ----------------------------------------------------------------------------- head
 def _bf16(x):
     return torch.from_numpy(np.asarray(x, np.float32)).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
