@@ -73,7 +73,6 @@ int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_
     if (e == cudaSuccess) e = cudaMalloc(&ctx->tasks, (size_t)max_B * sizeof(int2));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->task_ctl, 8 * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->task_ctl, 0, 8 * sizeof(int32_t));
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->task_rec, 2 * (size_t)max_B * sizeof(float4));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->task_ready, (size_t)max_B * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->task_ready, 0, (size_t)max_B * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->flags, 0, nflag * sizeof(int32_t));
@@ -106,7 +105,6 @@ int specdec_destroy(specdec_ctx* ctx) {
     cudaFree(ctx->norms);
     cudaFree(ctx->tasks);
     cudaFree(ctx->task_ctl);
-    cudaFree(ctx->task_rec);
     cudaFree(ctx->task_ready);
     cudaFree(ctx->stage);
     cudaFree(ctx->act[0]);
@@ -144,8 +142,9 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
         return fail(ctx, SPECDEC_EINVAL, "verify_correct: row_stats must be 16-byte aligned");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     ctx->epoch = (ctx->epoch + 1) & 0x3fffffffu;
-    if (ctx->epoch == 0) {   // wrapped: forget every stale flag before reusing epoch numbers
+    if ((ctx->epoch & 0xffffffu) == 0)   // the row records carry 24 epoch bits
         CU(ctx, cudaMemsetAsync(ctx->task_ready, 0, (size_t)ctx->max_B * sizeof(int32_t), s));
+    if (ctx->epoch == 0) {   // wrapped: forget every stale flag before reusing epoch numbers
         CU(ctx, cudaMemsetAsync(ctx->flags, 0, (size_t)ctx->max_B * ctx->max_K * sizeof(int32_t), s));
         ctx->epoch = 1;
     }
@@ -172,7 +171,6 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
     p.norms = ctx->norms;
     p.tasks = ctx->tasks;
     p.task_ctl = ctx->task_ctl;
-    p.task_rec = ctx->task_rec;
     p.task_ready = ctx->task_ready;
     p.epoch = ctx->epoch;
 
@@ -184,6 +182,7 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
         const double bytes = 2.0 * B * (K + 1.0) * V * (dtype == SPECDEC_BF16 ? 2 : 4);
         kind = (stream_ok && bytes >= 512e6) ? SPECDEC_VERIFY_FUSED : SPECDEC_VERIFY_DIRECT;
     }
+    if (kind == SPECDEC_VERIFY_FUSED && K > 63) kind = SPECDEC_VERIFY_STREAM;     // row records hold n in 6 bits
     if (kind != SPECDEC_VERIFY_DIRECT && !stream_ok)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: streaming kernels need 16-byte aligned rows (V=%d)", V);
     int n_launch = 0;
@@ -207,8 +206,9 @@ int specdec_verify_greedy(specdec_ctx* ctx, const void* target_logits, specdec_d
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_greedy: B=%d K=%d exceed the context (max_B=%d max_K=%d)", B, K, ctx->max_B, ctx->max_K);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     ctx->epoch = (ctx->epoch + 1) & 0x3fffffffu;
-    if (ctx->epoch == 0) {
+    if ((ctx->epoch & 0xffffffu) == 0)
         CU(ctx, cudaMemsetAsync(ctx->task_ready, 0, (size_t)ctx->max_B * sizeof(int32_t), s));
+    if (ctx->epoch == 0) {
         CU(ctx, cudaMemsetAsync(ctx->flags, 0, (size_t)ctx->max_B * ctx->max_K * sizeof(int32_t), s));
         ctx->epoch = 1;
     }

@@ -208,7 +208,6 @@ extern "C" int specdec_verify_correct_static(const void* target_logits, const vo
     p.norms = nullptr;
     p.tasks = nullptr;
     p.task_ctl = nullptr;
-    p.task_rec = nullptr;
     p.task_ready = nullptr;
     p.epoch = epoch;
     e = dtype == SPECDEC_BF16 ? launch_static<__nv_bfloat16>(p, s) : launch_static<float>(p, s);

@@ -459,12 +459,12 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) verify_stream_draw_kernel(c
 
 // =============================================================================================
 // Fused kernel: the same pipeline in one launch.  Phase 1 is the statistics pass above.  Every row
-// of the batch ends in exactly one record in a global queue -- {b, n, mode, u, normalisers},
-// written by the epilogue warp that resolves the row (mode 0 for rows that draw nothing: bad
-// length or bad token) and stamped ready with the call's epoch.  When a CTA's producer has
-// streamed its last unit it turns to the queue: it claims record t = head++, waits (bounded) for
-// its stamp, and streams that row pair through the same ring as a draw unit, described to the
-// worker and epilogue warps by a small descriptor ring in shared memory; t >= B ends the CTA.
+// of the batch ends in exactly one record, a single word {epoch, mode, n} stored (release) by the
+// epilogue warp that resolves the row (mode 0 for rows that draw nothing: bad length or bad
+// token).  When a CTA's producer has streamed its last unit it claims rows in order (head++),
+// waits (bounded) for the row's record, fetches the row's normalisers and uniform, and streams
+// that row pair through the same ring as a draw unit, described to the
+// worker and epilogue warps by a small descriptor ring in shared memory; a claim >= B ends the CTA.
 // Draws are therefore spread over all CTAs dynamically, overlap the tail of the statistics pass,
 // and find their rows in L2 whenever the batch fits there.  CTAs only ever wait for records of
 // rows whose units belong to CTAs of the same launch (grid <= SM count, one CTA per SM).
@@ -485,19 +485,13 @@ struct FusedShared {
     DrawDesc desc[DQ];
 };
 
-// One queue record for row b (called by one lane).
+// The record of row b (called by one lane): a single word {epoch, mode, n}, so that publishing it
+// is one release store and reading it needs no second access.
+__device__ __forceinline__ int record_stamp(uint32_t epoch, int mode, int n) {
+    return (int)(((epoch & 0xffffffu) << 8) | ((uint32_t)mode << 6) | (uint32_t)n);
+}
 __device__ __forceinline__ void push_record(const VerifyParams& P, int b, int n, int mode) {
-    float4 nv = make_float4(0.f, 0.f, 0.f, 0.f);
-    float u01 = 0.f;
-    if (mode) {
-        nv = __ldcg(&P.norms[(size_t)b * (P.K + 1) + n]);
-        u01 = P.uniforms[(size_t)b * (P.K + 1) + P.K];
-    }
-    const int t = atomicAdd(&P.task_ctl[2], 1);
-    P.task_rec[2 * t] = make_float4(__int_as_float(b), __int_as_float(n), __int_as_float(mode), u01);
-    P.task_rec[2 * t + 1] = nv;
-    __threadfence();
-    st_release(&P.task_ready[t], (int)P.epoch);
+    st_release(&P.task_ready[b], record_stamp(P.epoch, mode, mode ? n : 0));
 }
 
 // next_unit for the fused kernel's reporting warp: a row with a bad length also gets its record.
@@ -573,20 +567,24 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) verify_fused_kernel(const V
         // ---- phase 2: draws from the global queue
         uint32_t seq2 = 0;
         for (;;) {
-            const int t = atomicAdd(&P.task_ctl[3], 1);
-            if (t >= P.B) break;
+            const int b = atomicAdd(&P.task_ctl[3], 1);          // rows are claimed in order
+            if (b >= P.B) break;
+            uint32_t stamp = 0;
             bool ok = false;
-            for (uint32_t it = 0; it < RECORD_POLLS && !(ok = (ld_acquire(&P.task_ready[t]) == (int)P.epoch)); ++it)
+            for (uint32_t it = 0; it < RECORD_POLLS; ++it) {
+                stamp = (uint32_t)ld_acquire(&P.task_ready[b]);
+                if ((ok = ((stamp >> 8) == (P.epoch & 0xffffffu)))) break;
                 __nanosleep(200);
+            }
             if (!ok) { atomicOr(P.status, SPECDEC_DATA_WAIT_LIMIT); continue; }
-            const float4 r0 = __ldcg(&P.task_rec[2 * t]), r1 = __ldcg(&P.task_rec[2 * t + 1]);
-            const int mode = __float_as_int(r0.z);
+            const int mode = (int)((stamp >> 6) & 3u), n = (int)(stamp & 63u);
             if (mode == 0) continue;
-            const int b = __float_as_int(r0.x), n = __float_as_int(r0.y);
+            const float4 r1 = __ldcg(&P.norms[(size_t)b * (P.K + 1) + n]);
+            const float u01 = __ldcg(&P.uniforms[(size_t)b * (P.K + 1) + P.K]);
             // the descriptor must be in place before the unit's first tile can complete
             mbar_wait(smem_u32(&ss.empty[stage]), phase ^ 1u, P.status);
             DrawDesc& d = fs.desc[seq2 % DQ];
-            d.kind = mode; d.b = b; d.n = n; d.u01 = r0.w;
+            d.kind = mode; d.b = b; d.n = n; d.u01 = u01;
             d.np = Norm{r1.x, r1.y}; d.nq = Norm{r1.z, r1.w};
             produce_unit(ss, ring, tbase + ((size_t)b * (P.K + 1) + n) * row_bytes,
                          dbase + ((size_t)b * P.K + n) * row_bytes, mode == 2, row_bytes, ntiles, stage, phase, P.status);
@@ -599,7 +597,6 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) verify_fused_kernel(const V
         // the last producer to finish empties the queue counters for the next call
         __threadfence();
         if (atomicAdd(&P.task_ctl[4], 1) == (int)gridDim.x - 1) {
-            P.task_ctl[2] = 0;
             P.task_ctl[3] = 0;
             P.task_ctl[4] = 0;
         }
