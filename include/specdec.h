@@ -203,6 +203,15 @@ int specdec_stop_step(specdec_ctx* ctx, const float* accept_prob_step, float* p_
                       int32_t* stop, void* stream);
 
 /*
+ * Self-test of the kernels' failure handling (no counterpart in the paper).  Every in-kernel wait
+ * of this library is bounded: when it runs out the kernel sets SPECDEC_DATA_WAIT_LIMIT in the
+ * status word and carries on instead of hanging.  This call launches a one-thread kernel that
+ * waits, with a budget of 4096 polls, on a barrier nothing will ever complete; afterwards
+ * specdec_device_status() must report SPECDEC_DATA_WAIT_LIMIT and the context must still work.
+ */
+int specdec_selftest_wait_limit(specdec_ctx* ctx, void* stream);
+
+/*
  * Allocation-free variant of specdec_verify_correct.  The paper has no counterpart: this entry
  * point exists for callers that cannot call cudaMalloc -- a serving process that has given all
  * device memory to its own pool, a plugin whose host forbids allocations after start-up, a

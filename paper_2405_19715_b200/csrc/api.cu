@@ -305,4 +305,12 @@ int specdec_stop_step(specdec_ctx* ctx, const float* accept_prob_step, float* p_
     return SPECDEC_OK;
 }
 
+int specdec_selftest_wait_limit(specdec_ctx* ctx, void* stream) {
+    if (!ctx) return SPECDEC_EINVAL;
+    cudaError_t e = launch_wait_limit_selftest(ctx->status, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "selftest launch");
+    ctx->launches += 1;
+    return SPECDEC_OK;
+}
+
 }  // extern "C"

@@ -802,6 +802,19 @@ cudaError_t launch_fused_t(const VerifyParams& p, int sm_count, size_t smem, cud
     return cudaGetLastError();
 }
 
+// Self-test of the bounded waits: one thread waits on an mbarrier that nothing will ever complete,
+// with a small poll budget, and must come back with SPECDEC_DATA_WAIT_LIMIT set.
+__global__ void wait_limit_selftest_kernel(uint32_t* status, uint32_t polls) {
+    __shared__ unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        bool ok = false;
+        for (uint32_t it = 0; it < polls && !(ok = mbar_try_wait(smem_u32(&bar), 0)); ++it) {}
+        if (!ok) atomicOr(status, SPECDEC_DATA_WAIT_LIMIT);
+    }
+}
+
 size_t stream_smem(int V, int elem_size) {
     const int epv = 16 / elem_size;
     const int nslab = ((V + epv - 1) / epv + 31) / 32;
@@ -845,4 +858,9 @@ cudaError_t launch_verify_stream(const VerifyParams& p, specdec_dtype dtype, int
     const int es = dtype == SPECDEC_BF16 ? 2 : 4;
     const size_t smem = stream_smem(p.V, es);
     return dtype == SPECDEC_BF16 ? launch_t<__nv_bfloat16>(p, sm_count, smem, s) : launch_t<float>(p, sm_count, smem, s);
+}
+
+cudaError_t launch_wait_limit_selftest(uint32_t* status, cudaStream_t s) {
+    wait_limit_selftest_kernel<<<1, 32, 0, s>>>(status, 4096u);
+    return cudaGetLastError();
 }

@@ -19,7 +19,7 @@ DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT = 1, 2, 4
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
            "specdec_launch_count", "specdec_verify_correct", "specdec_verify_correct_host",
-           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step"]
+           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step", "specdec_selftest_wait_limit"]
 STATIC_MAX_UNITS, STATIC_MAX_V = 16384, 262144
 
 
@@ -58,6 +58,7 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
                                                 C.c_int, C.c_int, ip, ip, fp, C.c_uint32, C.c_void_p]
     lib.specdec_accept_head.argtypes = [C.c_void_p, vp, C.POINTER(_Head), C.c_int, C.c_int, fp, C.c_void_p]
     lib.specdec_stop.argtypes = [C.c_void_p, fp, ip, C.c_float, C.c_int, C.c_int, ip, C.c_void_p]
+    lib.specdec_selftest_wait_limit.argtypes = [C.c_void_p, C.c_void_p]
     lib.specdec_stop_step.argtypes = [C.c_void_p, fp, fp, C.c_float, C.c_int, ip, C.c_void_p]
     lib.specdec_verify_greedy.argtypes = [C.c_void_p, vp, C.c_int, ip, ip, C.c_int, C.c_int, C.c_int, ip, ip, ip,
                                           C.c_void_p]
@@ -187,6 +188,11 @@ def specdec_verify_correct_host(ctx: Context, target_logits, draft_logits, cand_
         _ptr(accept_ratio, torch.float32, False), flags, _stream(stream))
     ctx._check(rc)
     return n_accepted, next_token
+
+
+def specdec_selftest_wait_limit(ctx: Context, stream=None):
+    """specdec_selftest_wait_limit of the C ABI (sets the WAIT_LIMIT status bit by design)."""
+    ctx._check(ctx.lib.specdec_selftest_wait_limit(ctx.handle, _stream(stream)))
 
 
 def specdec_stop_step(ctx: Context, accept_prob_step, p_hat, h: float, stop=None, stream=None):

@@ -234,3 +234,26 @@ def test_stop_rule_parity(ctx):
     pos = specdec.specdec_stop(specdec.Context(3000, 20), torch.from_numpy(big).cuda(), 0.6).cpu().numpy()
     rep = parity.classify_stop(big, 0.6, pos)
     assert rep["exact"] + rep["boundary"] == 3000
+
+
+def test_bounded_wait_reports_and_context_survives(ctx):
+    """A wait that can never complete ends by itself, sets the status bit, and leaves the context usable."""
+    specdec.specdec_selftest_wait_limit(ctx)
+    assert ctx.device_status() == specdec.DATA_WAIT_LIMIT
+    assert ctx.device_status() == 0
+    cfg = wl.CONFIGS["cfg2"]
+    inp = wl.make_verify_inputs(cfg)
+    for flags in KERNELS:
+        parity.classify_rows(inp, parity.run_gpu_verify(ctx, inp, flags), dtype="f32")
+    assert ctx.device_status() == 0
+
+
+@pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
+def test_wide_shapes(ctx, flags):
+    """K = 32 (the ballot's full width), a batch larger than the SM count, a vocabulary of 262144."""
+    for B, K, V, dtype in ((200, 32, 2048, "bf16"), (3, 2, 262144, "bf16"), (2, 3, 100000, "f32")):
+        cfg = wl.Workload("wide", B=B, K=K, V=V, dtype=dtype, sigma_d=3.0, sigma_n=1.0, T=0.9, ragged=True, seed=B + V)
+        inp = wl.make_verify_inputs(cfg)
+        gpu = parity.run_gpu_verify(ctx, inp, flags)
+        rep = parity.classify_rows(inp, gpu, dtype="f32")
+        assert rep["rows"] == B and ctx.device_status() == 0
