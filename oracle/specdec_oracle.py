@@ -41,7 +41,7 @@ import numpy as np
 __all__ = [
     "bf16_bits_to_f64", "logits_to_f64", "softmax_T", "log_sum_exp_T",
     "accept_ratio", "first_rejection", "residual", "inverse_cdf",
-    "verify_from_probs", "verify_correct", "sampling_weights",
+    "verify_from_probs", "verify_correct", "sampling_weights", "top_k_filter",
     "silu", "sigmoid", "accept_head", "stop_rule", "greedy_verify", "greedy_verify_tokens", "stop_step",
 ]
 
@@ -88,6 +88,17 @@ def log_sum_exp_T(z: np.ndarray, T) -> np.ndarray:
     x = np.asarray(z, dtype=np.float64) / _temperature(T)
     m = np.max(x, axis=-1, keepdims=True)
     return (m + np.log(np.sum(np.exp(x - m), axis=-1, keepdims=True)))[..., 0]
+
+
+def top_k_filter(z: np.ndarray, k) -> np.ndarray:
+    """Top-k sampling filter (Appendix D.1: the paper samples with k = 50): logits below the k-th
+    largest of the row become -inf, so their probability is zero; ties with the k-th largest are
+    kept.  k = None or k >= V leaves the row unchanged."""
+    z = np.asarray(z, dtype=np.float64)
+    if k is None or k >= z.shape[-1]:
+        return z
+    kth = np.sort(z, axis=-1)[..., -int(k)][..., None]
+    return np.where(z >= kth, z, -np.inf)
 
 
 # --------------------------------------------------------------------------- one rejection step
@@ -154,19 +165,20 @@ def verify_from_probs(p, q, y, L: int, r, u):
 
 
 # --------------------------------------------------------------------------- batched, from logits
-def sampling_weights(target_row, draft_row, T):
+def sampling_weights(target_row, draft_row, T, top_k=None):
     """Un-normalised weights y' is drawn from at one position: (p - q)_+ when a draft
-    row is given (rejection), p itself when ``draft_row`` is None (bonus)."""
-    p = softmax_T(logits_to_f64(target_row), T)
+    row is given (rejection), p itself when ``draft_row`` is None (bonus).  With ``top_k`` both
+    distributions are the top-k filtered ones."""
+    p = softmax_T(top_k_filter(logits_to_f64(target_row), top_k), T)
     if draft_row is None:
         return p
-    w = residual(p, softmax_T(logits_to_f64(draft_row), T))
+    w = residual(p, softmax_T(top_k_filter(logits_to_f64(draft_row), top_k), T))
     if not (np.cumsum(w)[-1] > 1e-30):
         return p
     return w
 
 
-def verify_correct(target_logits, draft_logits, cand_tokens, cand_len, uniforms, T):
+def verify_correct(target_logits, draft_logits, cand_tokens, cand_len, uniforms, T, top_k=None):
     """Batched verify + correct (Algorithm 2, lower half of Algorithm 1).
 
     target_logits [B,K+1,V], draft_logits [B,K,V] (float32 or uint16 bf16 bits),
@@ -199,24 +211,29 @@ def verify_correct(target_logits, draft_logits, cand_tokens, cand_len, uniforms,
             y = int(cand_tokens[b, i])
             if not (0 <= y < V):
                 raise ValueError(f"cand_tokens[{b},{i}]={y} outside [0,{V})")
-            t = logits_to_f64(target_logits[b, i])
-            d = logits_to_f64(draft_logits[b, i])
+            t = top_k_filter(logits_to_f64(target_logits[b, i]), top_k)
+            d = top_k_filter(logits_to_f64(draft_logits[b, i]), top_k)
             lp, lq = log_sum_exp_T(t, T), log_sum_exp_T(d, T)
             log_py, log_qy = t[y] / T - lp, d[y] / T - lq
-            ratio = np.exp(log_py - log_qy)          # = p_i(y_i) / q_i(y_i)
+            if log_py == -np.inf:                    # p_i(y_i) = 0 (filtered out): certain rejection
+                ratio = 0.0
+            elif log_qy == -np.inf:                  # q_i(y_i) = 0 < p_i(y_i)
+                ratio = np.inf
+            else:
+                ratio = np.exp(log_py - log_qy)      # = p_i(y_i) / q_i(y_i)
             ratios.append(ratio)
             out["lse_p"][b, i], out["lse_q"][b, i] = lp, lq
             out["p_y"][b, i], out["q_y"][b, i] = np.exp(log_py), np.exp(log_qy)
             out["accept_ratio"][b, i] = min(1.0, ratio)
         n = first_rejection(ratios, uniforms[b, :K], L)
         if n < L:
-            w = sampling_weights(target_logits[b, n], draft_logits[b, n], T)
-            pn = softmax_T(logits_to_f64(target_logits[b, n]), T)
-            qn = softmax_T(logits_to_f64(draft_logits[b, n]), T)
+            w = sampling_weights(target_logits[b, n], draft_logits[b, n], T, top_k)
+            pn = softmax_T(top_k_filter(logits_to_f64(target_logits[b, n]), top_k), T)
+            qn = softmax_T(top_k_filter(logits_to_f64(draft_logits[b, n]), top_k), T)
             out["resid_mass"][b] = np.cumsum(residual(pn, qn))[-1]
         else:
-            out["lse_p"][b, L] = log_sum_exp_T(logits_to_f64(target_logits[b, L]), T)
-            w = sampling_weights(target_logits[b, L], None, T)
+            out["lse_p"][b, L] = log_sum_exp_T(top_k_filter(logits_to_f64(target_logits[b, L]), top_k), T)
+            w = sampling_weights(target_logits[b, L], None, T, top_k)
             out["resid_mass"][b] = 1.0
         out["n_accepted"][b] = n
         out["next_token"][b] = inverse_cdf(w, uniforms[b, K])

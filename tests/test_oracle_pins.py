@@ -444,6 +444,41 @@ def test_head_against_torch_float64_modules():
     assert not np.allclose(orc.accept_head(x, [(Ws[0].T.copy(), bs[0]), (Ws[1], bs[1])], w, -0.5), want, rtol=1e-3)
 
 
+def test_top_k_filter_against_torch_topk_and_its_limits():
+    """Appendix D.1's top-k sampling: the kept set is {v : z_v >= k-th largest} (library: torch.topk);
+    k >= V changes nothing; k = 1 turns the stochastic algorithm into the greedy one of Section 4.1."""
+    rng = np.random.default_rng(31)
+    z = np.round(rng.normal(scale=2, size=(6, 200)) * 4) / 4           # quarter steps: ties at the threshold occur
+    for k in (1, 5, 50, 199):
+        kth = torch.topk(torch.from_numpy(z), k, dim=-1).values[:, -1:].numpy()
+        want = np.where(z >= kth, z, -np.inf)
+        got = orc.top_k_filter(z, k)
+        assert np.array_equal(got, want)
+        assert np.all((got > -np.inf).sum(-1) >= k)
+    assert np.array_equal(orc.top_k_filter(z, 200), z) and np.array_equal(orc.top_k_filter(z, None), z)
+    B, K, V = 10, 4, 64
+    d = rng.normal(scale=2, size=(B, K, V)).astype(np.float32)
+    t = np.concatenate([d, d[:, :1]], 1) + rng.normal(scale=1.5, size=(B, K + 1, V)).astype(np.float32)
+    y = d.argmax(-1).astype(np.int32)
+    u = rng.random((B, K + 1)).astype(np.float32)
+    full = orc.verify_correct(t, d, y, None, u, 0.9)
+    same = orc.verify_correct(t, d, y, None, u, 0.9, top_k=V)
+    assert np.array_equal(full["n_accepted"], same["n_accepted"]) and np.array_equal(full["next_token"], same["next_token"])
+    one = orc.verify_correct(t, d, y, None, u, 0.9, top_k=1)
+    n_g, tok_g = orc.greedy_verify(t, d)
+    assert np.array_equal(one["n_accepted"], n_g) and np.array_equal(one["next_token"], tok_g)
+    # a drafted token outside the target's top-k is rejected with certainty; the draw stays inside it
+    k = 5
+    o = orc.verify_correct(t, d, y, None, u, 0.9, top_k=k)
+    for b in range(B):
+        n = o["n_accepted"][b]
+        keep = np.argsort(-t[b, n].astype(np.float64), kind="stable")[:k]
+        assert o["next_token"][b] in keep
+        for i in range(K):
+            if y[b, i] not in np.argsort(-t[b, i].astype(np.float64), kind="stable")[:k]:
+                assert o["accept_ratio"][b, i] == 0.0
+
+
 def test_greedy_case_is_the_low_temperature_limit():
     """Section 4.1: with greedy drafts the algorithm keeps candidates while they equal the target's
     argmax and emits the target's argmax at the first mismatch."""
