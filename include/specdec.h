@@ -51,6 +51,7 @@ typedef enum {
 #define SPECDEC_DATA_BAD_LENGTH 1u /* some cand_len[b] outside [0,K]                     */
 #define SPECDEC_DATA_BAD_TOKEN  2u /* some cand_tokens[b,i] outside [0,V)                */
 #define SPECDEC_DATA_WAIT_LIMIT 4u /* a bounded in-kernel wait gave up (outputs invalid) */
+#define SPECDEC_DATA_TOPK_TIES  8u /* top-k: thousands of logits tie with a row's k-th largest    */
 
 /* Kernel selection for specdec_verify_correct (flags argument). 0 lets the library pick. */
 #define SPECDEC_VERIFY_AUTO    0u
@@ -123,6 +124,26 @@ int specdec_verify_correct(specdec_ctx* ctx,
                            int32_t* n_accepted, int32_t* next_token,
                            float* accept_ratio, float* row_stats, float* resid_mass,
                            uint32_t flags, void* stream);
+
+/*
+ * Verify and correct under top-k sampling (Appendix D.1: the paper decodes with top-k sampling,
+ * k = 50).  In every row of both models the logits below the row's k-th largest value count as
+ * -inf (ties with the k-th largest are kept); Algorithm 2 then runs on the filtered distributions
+ * exactly as in specdec_verify_correct.  A drafted token outside the target's kept set is rejected
+ * with certainty; y' always lies in the target's kept set.  top_k >= V is the unfiltered
+ * operation.  Arguments as for specdec_verify_correct; 1 <= top_k <= 256 (or >= V).
+ * The kept logits' probabilities are evaluated in fp64.  Logits equal to the k-th largest are all
+ * kept.  Where more than 2048 logits of a target row, or 4096 of a draft row, are kept that way the
+ * call sets SPECDEC_DATA_TOPK_TIES: an accept test it touches reports n_accepted = -1, a draw it
+ * touches next_token = -1.
+ */
+int specdec_verify_correct_topk(specdec_ctx* ctx,
+                                const void* target_logits, const void* draft_logits, specdec_dtype dtype,
+                                const int32_t* cand_tokens, const int32_t* cand_len,
+                                const float* uniforms, float temperature, int top_k,
+                                int B, int K, int V,
+                                int32_t* n_accepted, int32_t* next_token,
+                                float* accept_ratio, float* resid_mass, void* stream);
 
 /*
  * Greedy verification (Section 4.1: the deterministic setting in which both models decode

@@ -126,7 +126,7 @@ int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits) {
     CU(ctx, cudaMemsetAsync(ctx->status, 0, sizeof(uint32_t), s));
     CU(ctx, cudaStreamSynchronize(s));
     if (bits) *bits = host;
-    if (host) return fail(ctx, SPECDEC_EDATA, "device status bits 0x%x (1 = bad cand_len, 2 = bad token, 4 = wait limit)", host);
+    if (host) return fail(ctx, SPECDEC_EDATA, "device status bits 0x%x (1 = bad cand_len, 2 = bad token, 4 = wait limit, 8 = top-k ties)", host);
     return SPECDEC_OK;
 }
 
@@ -191,6 +191,53 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
                                                     : launch_verify_direct(p, dtype, s, &n_launch);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "verify_correct launch");
     ctx->launches += n_launch;
+    return SPECDEC_OK;
+}
+
+int specdec_verify_correct_topk(specdec_ctx* ctx, const void* target_logits, const void* draft_logits,
+                                specdec_dtype dtype, const int32_t* cand_tokens, const int32_t* cand_len,
+                                const float* uniforms, float temperature, int top_k, int B, int K, int V,
+                                int32_t* n_accepted, int32_t* next_token, float* accept_ratio, float* resid_mass,
+                                void* stream) {
+    if (ctx && top_k >= V && V >= 1)
+        return specdec_verify_correct(ctx, target_logits, draft_logits, dtype, cand_tokens, cand_len, uniforms,
+                                      temperature, B, K, V, n_accepted, next_token, accept_ratio, nullptr,
+                                      resid_mass, SPECDEC_VERIFY_AUTO, stream);
+    int rc = check_verify_args(ctx, target_logits, draft_logits, (int)dtype, cand_tokens, uniforms, temperature, B,
+                               K, V, n_accepted, next_token, SPECDEC_VERIFY_AUTO);
+    if (rc != SPECDEC_OK) return rc;
+    if (top_k < 1 || top_k > 256) return fail(ctx, SPECDEC_EINVAL, "verify_correct_topk: top_k must be in [1, 256] or >= V (got %d)", top_k);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    ctx->epoch = (ctx->epoch + 1) & 0x3fffffffu;
+    if ((ctx->epoch & 0xffffffu) == 0)
+        CU(ctx, cudaMemsetAsync(ctx->task_ready, 0, (size_t)ctx->max_B * sizeof(int32_t), s));
+    if (ctx->epoch == 0) {
+        CU(ctx, cudaMemsetAsync(ctx->flags, 0, (size_t)ctx->max_B * ctx->max_K * sizeof(int32_t), s));
+        ctx->epoch = 1;
+    }
+    VerifyParams p = {};
+    p.target = target_logits;
+    p.draft = draft_logits;
+    p.tokens = cand_tokens;
+    p.lens = cand_len;
+    p.uniforms = uniforms;
+    p.c = (float)(1.4426950408889634 / (double)temperature);
+    p.B = B;
+    p.K = K;
+    p.V = V;
+    p.n_acc = n_accepted;
+    p.next = next_token;
+    p.ratio = accept_ratio;
+    p.rmass = resid_mass;
+    p.flags = ctx->flags;
+    p.draws = ctx->draws;
+    p.draw_mass = ctx->draw_mass;
+    p.arrive = ctx->arrive;
+    p.status = ctx->status;
+    p.epoch = ctx->epoch;
+    cudaError_t e = launch_verify_topk(p, dtype, top_k, s);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "verify_correct_topk launch");
+    ctx->launches += 1;
     return SPECDEC_OK;
 }
 

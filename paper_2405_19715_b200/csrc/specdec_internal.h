@@ -69,3 +69,4 @@ cudaError_t launch_stop(const float* accept_prob, const int32_t* lens, float h, 
 cudaError_t launch_stop_step(const float* accept_prob_step, float* p_hat, float h, int B, int32_t* stop,
                              cudaStream_t s);
 cudaError_t launch_wait_limit_selftest(uint32_t* status, cudaStream_t s);
+cudaError_t launch_verify_topk(const VerifyParams& p, specdec_dtype dtype, int top_k, cudaStream_t s);

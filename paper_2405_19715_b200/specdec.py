@@ -15,11 +15,11 @@ from . import build as _build
 F32, BF16 = 0, 1
 OK, EINVAL, EUNSUPPORTED, ECUDA, EDATA = 0, 1, 2, 3, 4
 VERIFY_AUTO, VERIFY_DIRECT, VERIFY_STREAM, VERIFY_FUSED = 0, 1, 2, 3
-DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT = 1, 2, 4
+DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT, DATA_TOPK_TIES = 1, 2, 4, 8
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
            "specdec_launch_count", "specdec_verify_correct", "specdec_verify_correct_host",
-           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step", "specdec_selftest_wait_limit"]
+           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step", "specdec_selftest_wait_limit", "specdec_verify_correct_topk"]
 STATIC_MAX_UNITS, STATIC_MAX_V = 16384, 262144
 
 
@@ -58,6 +58,8 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
                                                 C.c_int, C.c_int, ip, ip, fp, C.c_uint32, C.c_void_p]
     lib.specdec_accept_head.argtypes = [C.c_void_p, vp, C.POINTER(_Head), C.c_int, C.c_int, fp, C.c_void_p]
     lib.specdec_stop.argtypes = [C.c_void_p, fp, ip, C.c_float, C.c_int, C.c_int, ip, C.c_void_p]
+    lib.specdec_verify_correct_topk.argtypes = [C.c_void_p, vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int, C.c_int,
+                                                C.c_int, C.c_int, ip, ip, fp, fp, C.c_void_p]
     lib.specdec_selftest_wait_limit.argtypes = [C.c_void_p, C.c_void_p]
     lib.specdec_stop_step.argtypes = [C.c_void_p, fp, fp, C.c_float, C.c_int, ip, C.c_void_p]
     lib.specdec_verify_greedy.argtypes = [C.c_void_p, vp, C.c_int, ip, ip, C.c_int, C.c_int, C.c_int, ip, ip, ip,
@@ -186,6 +188,25 @@ def specdec_verify_correct_host(ctx: Context, target_logits, draft_logits, cand_
         _ptr(uniforms, torch.float32, False), float(temperature), B, K, V,
         _ptr(n_accepted, torch.int32, False), _ptr(next_token, torch.int32, False),
         _ptr(accept_ratio, torch.float32, False), flags, _stream(stream))
+    ctx._check(rc)
+    return n_accepted, next_token
+
+
+def specdec_verify_correct_topk(ctx: Context, target_logits, draft_logits, cand_tokens, cand_len, uniforms,
+                                temperature: float, top_k: int, n_accepted=None, next_token=None, accept_ratio=None,
+                                resid_mass=None, stream=None):
+    """specdec_verify_correct_topk of the C ABI.  Returns (n_accepted, next_token) device tensors."""
+    B, K1, V = target_logits.shape
+    dev = target_logits.device
+    if n_accepted is None:
+        n_accepted = torch.empty(B, dtype=torch.int32, device=dev)
+    if next_token is None:
+        next_token = torch.empty(B, dtype=torch.int32, device=dev)
+    rc = ctx.lib.specdec_verify_correct_topk(
+        ctx.handle, _ptr(target_logits), _ptr(draft_logits), _logit_dtype(target_logits),
+        _ptr(cand_tokens, torch.int32), _ptr(cand_len, torch.int32), _ptr(uniforms, torch.float32),
+        float(temperature), int(top_k), B, K1 - 1, V, _ptr(n_accepted, torch.int32), _ptr(next_token, torch.int32),
+        _ptr(accept_ratio, torch.float32), _ptr(resid_mass, torch.float32), _stream(stream))
     ctx._check(rc)
     return n_accepted, next_token
 

@@ -46,7 +46,7 @@ def _cdf_interval(w, g):
     return lo, c[g] / tot, w[g]
 
 
-def classify_rows(inp, gpu, rows=None, dtype="bf16", check_probs=True):
+def classify_rows(inp, gpu, rows=None, dtype="bf16", check_probs=True, top_k=None):
     """Compare GPU outputs with the oracle on `rows` (default all).  Returns a report dict and
     raises AssertionError on any row that is neither exact nor boundary-valid."""
     tl, dl = inp["target_logits"], inp["draft_logits"]
@@ -56,7 +56,7 @@ def classify_rows(inp, gpu, rows=None, dtype="bf16", check_probs=True):
     T = inp["temperature"]
     lens = np.full(B, K, np.int32) if inp.get("cand_len") is None else np.asarray(inp["cand_len"])
     sub = np.array(rows)
-    o = orc.verify_correct(tl[sub], dl[sub], inp["cand_tokens"][sub], lens[sub], inp["uniforms"][sub], T)
+    o = orc.verify_correct(tl[sub], dl[sub], inp["cand_tokens"][sub], lens[sub], inp["uniforms"][sub], T, top_k=top_k)
     rep = dict(rows=len(rows), exact=0, boundary_n=0, boundary_token=0, max_ratio_rel=0.0, max_lse_abs=0.0,
                max_prob_rel=0.0, max_mass_rel=0.0)
     rtol = PROB_RTOL[dtype]
@@ -79,10 +79,10 @@ def classify_rows(inp, gpu, rows=None, dtype="bf16", check_probs=True):
             if gn < L and gn > m:
                 assert r[gn] >= ratios[gn] - BOUNDARY, f"row {b}: position {gn} rejected against the oracle"
             n_boundary = True
-            w = orc.sampling_weights(tl[b, gn], dl[b, gn] if gn < L else None, T)
+            w = orc.sampling_weights(tl[b, gn], dl[b, gn] if gn < L else None, T, top_k)
             ot = orc.inverse_cdf(w, u)                     # the oracle's draw at the GPU's n
         if gt != ot:
-            w = orc.sampling_weights(tl[b, gn], dl[b, gn] if gn < L else None, T)
+            w = orc.sampling_weights(tl[b, gn], dl[b, gn] if gn < L else None, T, top_k)
             lo, hi, wg = _cdf_interval(w, gt)
             assert wg > 0 and lo - BOUNDARY <= u <= hi + BOUNDARY, \
                 f"row {b}: token {gt} vs oracle {ot}: u={u!r} interval=({lo!r},{hi!r}) w={wg!r}"
@@ -91,6 +91,14 @@ def classify_rows(inp, gpu, rows=None, dtype="bf16", check_probs=True):
             rep["boundary_n"] += 1
         else:
             rep["exact"] += 1
+        if not check_probs and "accept_ratio" in gpu:       # entry points without row_stats: ratios and mass only
+            for i in range(L):
+                rel = abs(gpu["accept_ratio"][b, i] - ratios[i]) / max(ratios[i], 1e-30)
+                rep["max_ratio_rel"] = max(rep["max_ratio_rel"], rel if ratios[i] > 0 else abs(gpu["accept_ratio"][b, i]))
+                assert (rel <= rtol) if ratios[i] > 0 else gpu["accept_ratio"][b, i] == 0, \
+                    f"row {b} pos {i}: accept ratio {gpu['accept_ratio'][b, i]!r} vs {ratios[i]!r}"
+            if gn == on and "resid_mass" in gpu:
+                assert abs(gpu["resid_mass"][b] - o["resid_mass"][k]) <= rtol * o["resid_mass"][k] + 1e-6
         if check_probs and "accept_ratio" in gpu:
             ga, st = gpu["accept_ratio"][b], gpu["row_stats"][b]
             for i in range(L):
