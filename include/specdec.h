@@ -165,6 +165,20 @@ int specdec_verify_greedy(specdec_ctx* ctx, const void* target_logits, specdec_d
                           void* stream);
 
 /*
+ * Sampling one token per row from softmax(logits / temperature): the drafting step y_i ~ q_i of
+ * Algorithm 1 and, on the target's logits, the K = 0 case of Algorithm 2 (a round with no candidates
+ * draws y' ~ p_1).  The draw is the inverse CDF in vocabulary order at uniforms[b], the rule
+ * specdec_verify_correct uses for y', so a drafted token and a verification of it share one
+ * definition of "sample".  With 1 <= top_k <= 256 the row is first restricted to its top_k largest
+ * logits (ties with the k-th kept); top_k <= 0 or >= V samples from the whole vocabulary.
+ *
+ *   logits   dev [B, V] row-major, dtype;  uniforms dev [B] fp32 in [0,1);  tokens dev out [B] int32
+ * Errors as for specdec_verify_correct (B <= max_B).
+ */
+int specdec_sample(specdec_ctx* ctx, const void* logits, specdec_dtype dtype, const float* uniforms,
+                   float temperature, int top_k, int B, int V, int32_t* tokens, void* stream);
+
+/*
  * Same operation with HOST input and output buffers: copies the inputs to device staging
  * buffers owned by the context (allocated or grown on first use), runs the kernels, copies
  * n_accepted / next_token (and accept_ratio when not NULL) back and synchronises `stream`

@@ -240,6 +240,16 @@ def verify_correct(target_logits, draft_logits, cand_tokens, cand_len, uniforms,
     return out
 
 
+def sample(logits, uniforms, T, top_k=None):
+    """Algorithm 1's drafting draw y ~ softmax(logits / T) for every row of logits [B, V] (also the
+    K = 0 round of Algorithm 2 on the target's logits): inverse CDF in vocabulary order at
+    uniforms[b], after the top-k filter of Appendix D.1 when top_k is given."""
+    z = logits_to_f64(logits)
+    u = np.asarray(uniforms, dtype=np.float64).reshape(-1)
+    return np.array([inverse_cdf(sampling_weights(z[b], None, T, top_k), u[b]) for b in range(z.shape[0])],
+                    dtype=np.int64)
+
+
 def greedy_verify_tokens(target_logits, cand_tokens, cand_len=None):
     """Greedy special case (Section 4.1) with the drafted tokens given: a candidate is kept while
     it equals argmax p_i, the first mismatch is replaced by argmax p_i, and argmax p_L is appended

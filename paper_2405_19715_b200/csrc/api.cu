@@ -241,6 +241,55 @@ int specdec_verify_correct_topk(specdec_ctx* ctx, const void* target_logits, con
     return SPECDEC_OK;
 }
 
+int specdec_sample(specdec_ctx* ctx, const void* logits, specdec_dtype dtype, const float* uniforms, float temperature,
+                   int top_k, int B, int V, int32_t* tokens, void* stream) {
+    if (!ctx) return SPECDEC_EINVAL;
+    if (!logits || !uniforms || !tokens) return fail(ctx, SPECDEC_EINVAL, "sample: null pointer argument");
+    if ((int)dtype != SPECDEC_F32 && (int)dtype != SPECDEC_BF16) return fail(ctx, SPECDEC_EINVAL, "sample: unknown dtype %d", (int)dtype);
+    if (!(temperature > 0.f) || !std::isfinite(temperature)) return fail(ctx, SPECDEC_EINVAL, "sample: temperature must be positive and finite");
+    if (V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "sample: V=%d above 2^22", V);
+    if (B < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "sample: B and V must be >= 1 (got %d, %d)", B, V);
+    if (B > ctx->max_B) return fail(ctx, SPECDEC_EUNSUPPORTED, "sample: B=%d exceeds the context (max_B=%d)", B, ctx->max_B);
+    if (top_k > 256 && top_k < V) return fail(ctx, SPECDEC_EINVAL, "sample: top_k must be <= 256, or <= 0 / >= V for none (got %d)", top_k);
+    cudaError_t e0 = cudaSetDevice(ctx->device);
+    if (e0 != cudaSuccess) return cuda_fail(ctx, e0, "cudaSetDevice");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    ctx->epoch = (ctx->epoch + 1) & 0x3fffffffu;
+    if ((ctx->epoch & 0xffffffu) == 0)
+        CU(ctx, cudaMemsetAsync(ctx->task_ready, 0, (size_t)ctx->max_B * sizeof(int32_t), s));
+    if (ctx->epoch == 0) {
+        CU(ctx, cudaMemsetAsync(ctx->flags, 0, (size_t)ctx->max_B * ctx->max_K * sizeof(int32_t), s));
+        ctx->epoch = 1;
+    }
+    // Algorithm 2 with no candidates: every row is its own bonus position
+    VerifyParams p = {};
+    p.target = logits;
+    p.draft = logits;
+    p.uniforms = uniforms;
+    p.c = (float)(1.4426950408889634 / (double)temperature);
+    p.B = B;
+    p.K = 0;
+    p.V = V;
+    p.n_acc = reinterpret_cast<int32_t*>(ctx->tasks);      // always 0 here; not reported
+    p.next = tokens;
+    p.flags = ctx->flags;
+    p.draws = ctx->draws;
+    p.draw_mass = ctx->draw_mass;
+    p.arrive = ctx->arrive;
+    p.status = ctx->status;
+    p.norms = ctx->norms;
+    p.tasks = ctx->tasks;
+    p.task_ctl = ctx->task_ctl;
+    p.task_ready = ctx->task_ready;
+    p.epoch = ctx->epoch;
+    int n_launch = 1;
+    cudaError_t e = (top_k >= 1 && top_k < V) ? launch_verify_topk(p, dtype, top_k, s)
+                                              : launch_verify_direct(p, dtype, s, &n_launch);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "sample launch");
+    ctx->launches += n_launch;
+    return SPECDEC_OK;
+}
+
 int specdec_verify_greedy(specdec_ctx* ctx, const void* target_logits, specdec_dtype dtype,
                           const int32_t* cand_tokens, const int32_t* cand_len, int B, int K, int V,
                           int32_t* n_accepted, int32_t* next_token, int32_t* target_argmax, void* stream) {

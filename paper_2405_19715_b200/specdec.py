@@ -19,7 +19,7 @@ DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT, DATA_TOPK_TIES = 1, 2, 4, 8
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
            "specdec_launch_count", "specdec_verify_correct", "specdec_verify_correct_host",
-           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step", "specdec_selftest_wait_limit", "specdec_verify_correct_topk"]
+           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step", "specdec_selftest_wait_limit", "specdec_verify_correct_topk", "specdec_sample"]
 STATIC_MAX_UNITS, STATIC_MAX_V = 16384, 262144
 
 
@@ -60,6 +60,7 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
     lib.specdec_stop.argtypes = [C.c_void_p, fp, ip, C.c_float, C.c_int, C.c_int, ip, C.c_void_p]
     lib.specdec_verify_correct_topk.argtypes = [C.c_void_p, vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int, C.c_int,
                                                 C.c_int, C.c_int, ip, ip, fp, fp, C.c_void_p]
+    lib.specdec_sample.argtypes = [C.c_void_p, vp, C.c_int, fp, C.c_float, C.c_int, C.c_int, C.c_int, ip, C.c_void_p]
     lib.specdec_selftest_wait_limit.argtypes = [C.c_void_p, C.c_void_p]
     lib.specdec_stop_step.argtypes = [C.c_void_p, fp, fp, C.c_float, C.c_int, ip, C.c_void_p]
     lib.specdec_verify_greedy.argtypes = [C.c_void_p, vp, C.c_int, ip, ip, C.c_int, C.c_int, C.c_int, ip, ip, ip,
@@ -209,6 +210,17 @@ def specdec_verify_correct_topk(ctx: Context, target_logits, draft_logits, cand_
         _ptr(accept_ratio, torch.float32), _ptr(resid_mass, torch.float32), _stream(stream))
     ctx._check(rc)
     return n_accepted, next_token
+
+
+def specdec_sample(ctx: Context, logits, uniforms, temperature: float, top_k: int = 0, tokens=None, stream=None):
+    """specdec_sample of the C ABI: logits [B, V], uniforms [B] -> tokens [B] int32 (device)."""
+    B, V = logits.shape
+    if tokens is None:
+        tokens = torch.empty(B, dtype=torch.int32, device=logits.device)
+    rc = ctx.lib.specdec_sample(ctx.handle, _ptr(logits), _logit_dtype(logits), _ptr(uniforms, torch.float32),
+                                float(temperature), int(top_k), B, V, _ptr(tokens, torch.int32), _stream(stream))
+    ctx._check(rc)
+    return tokens
 
 
 def specdec_selftest_wait_limit(ctx: Context, stream=None):

@@ -516,3 +516,18 @@ def test_pins_catch_planted_mistakes(monkeypatch):
         real = orc.inverse_cdf
         m.setattr(orc, "inverse_cdf", lambda w, u: min(real(w, u) + 1, len(w) - 1))
         assert not law_ok()
+
+
+def test_sample_law_on_a_dyadic_distribution():
+    """Algorithm 1's draw y ~ q: with q = (1/8, 1/2, 1/4, 1/8) and u swept over the midpoints of a
+    64-cell grid, every CDF breakpoint is a grid line, so the counts per token are exactly 64 q."""
+    q = np.array([1 / 8, 1 / 2, 1 / 4, 1 / 8])
+    u = (np.arange(64) + 0.5) / 64
+    logits = np.tile(np.log(q) * 0.7 + 3.0, (64, 1))          # temperature and shift must cancel
+    tok = orc.sample(logits, u, 0.7)
+    assert np.bincount(tok, minlength=4).tolist() == [8, 32, 16, 8]
+    assert np.all(np.diff(tok) >= 0)                           # vocabulary order
+    # top-2 keeps tokens 1 and 2 with probabilities 2/3, 1/3 -> 96 cells: 64, 32
+    u3 = (np.arange(96) + 0.5) / 96
+    tok2 = orc.sample(np.tile(np.log(q), (96, 1)), u3, 1.0, top_k=2)
+    assert np.bincount(tok2, minlength=4).tolist() == [0, 64, 32, 0]
