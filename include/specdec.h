@@ -179,6 +179,55 @@ int specdec_sample(specdec_ctx* ctx, const void* logits, specdec_dtype dtype, co
                    float temperature, int top_k, int B, int V, int32_t* tokens, void* stream);
 
 /*
+ * Verify/correct on logits split along the vocabulary (what a tensor-parallel output layer
+ * produces; the paper shards its 70B target over several GPUs, Appendix D.1).  Rank r of n_shards
+ * holds columns [v_offset, v_offset + V_shard) of both models' logits for all B rows.  Algorithm 2
+ * then needs two small exchanges, which the CALLER performs between three local calls (any
+ * all-gather will do; nothing here touches another GPU's memory or waits for another rank):
+ *
+ *   1. specdec_shard_stats   -> stats [B, K+1, 8] fp32 per rank; all-gather -> stats_all [n_shards, B, K+1, 8]
+ *   2. specdec_shard_accept  -> n_accepted (identical on every rank), row_norm, and this rank's
+ *                               mass [B] fp64 of the weights y' is drawn from; all-gather -> mass_all [n_shards, B]
+ *   3. specdec_shard_draw    -> next_token[b] on the one rank whose columns contain the draw, -1 on
+ *                               the others; a max-reduction over ranks yields next_token.
+ *
+ * The results equal specdec_verify_correct on the concatenated logits up to fp32 summation order.
+ * cand_tokens hold global token ids; V is the whole vocabulary (range check).  A drafted token that
+ * no rank, or more than one, holds marks the row bad (n_accepted = next_token = -1).
+ * n_shards <= SPECDEC_SHARD_MAX_RANKS.  All pointers are device memory; mass / mass_all are fp64.
+ */
+#define SPECDEC_SHARD_STATS_WIDTH 8
+#define SPECDEC_SHARD_MAX_RANKS 64
+typedef struct specdec_shard {
+    const void* target_logits;  /* dev [B, K+1, V_shard] row-major */
+    const void* draft_logits;   /* dev [B, K,   V_shard]           */
+    specdec_dtype dtype;
+    int V_shard;                /* columns held by this rank        */
+    int v_offset;               /* global token id of local column 0 */
+    int V;                      /* size of the whole vocabulary     */
+} specdec_shard;
+
+int specdec_shard_stats(specdec_ctx* ctx, const specdec_shard* shard,
+                        const int32_t* cand_tokens, const int32_t* cand_len, float temperature,
+                        int B, int K, float* stats, void* stream);
+int specdec_shard_accept(specdec_ctx* ctx, const specdec_shard* shard,
+                         const float* stats_all, int n_shards,
+                         const int32_t* cand_len, const float* uniforms, float temperature,
+                         int B, int K,
+                         int32_t* n_accepted,   /* dev out [B]                                  */
+                         float* accept_ratio,   /* dev out [B, K] or NULL                       */
+                         float* row_norm,       /* dev out [B, 4], 16-byte aligned: input of _draw */
+                         double* mass,          /* dev out [B]                                  */
+                         void* stream);
+int specdec_shard_draw(specdec_ctx* ctx, const specdec_shard* shard,
+                       const float* stats_all, const double* mass_all, int n_shards, int rank,
+                       const int32_t* n_accepted, const int32_t* cand_len, const float* uniforms,
+                       const float* row_norm, float temperature, int B, int K,
+                       int32_t* next_token,     /* dev out [B]: -1 unless this rank draws the row */
+                       float* resid_mass,       /* dev out [B] or NULL                            */
+                       void* stream);
+
+/*
  * Same operation with HOST input and output buffers: copies the inputs to device staging
  * buffers owned by the context (allocated or grown on first use), runs the kernels, copies
  * n_accepted / next_token (and accept_ratio when not NULL) back and synchronises `stream`

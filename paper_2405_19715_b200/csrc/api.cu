@@ -290,6 +290,72 @@ int specdec_sample(specdec_ctx* ctx, const void* logits, specdec_dtype dtype, co
     return SPECDEC_OK;
 }
 
+namespace {
+int check_shard_args(specdec_ctx* ctx, const specdec_shard* sh, float T, int B, int K, const char* who) {
+    if (!ctx) return SPECDEC_EINVAL;
+    if (!sh || !sh->target_logits || !sh->draft_logits) return fail(ctx, SPECDEC_EINVAL, "%s: null shard or logits", who);
+    if ((int)sh->dtype != SPECDEC_F32 && (int)sh->dtype != SPECDEC_BF16) return fail(ctx, SPECDEC_EINVAL, "%s: unknown dtype %d", who, (int)sh->dtype);
+    if (B < 1 || K < 1) return fail(ctx, SPECDEC_EINVAL, "%s: B and K must be >= 1 (got %d, %d)", who, B, K);
+    if (sh->V_shard < 1 || sh->v_offset < 0 || sh->V < 1 || (long long)sh->v_offset + sh->V_shard > (long long)sh->V)
+        return fail(ctx, SPECDEC_EINVAL, "%s: columns [%d, %d + %d) do not lie in a vocabulary of %d", who, sh->v_offset, sh->v_offset, sh->V_shard, sh->V);
+    if (!(T > 0.f) || !std::isfinite(T)) return fail(ctx, SPECDEC_EINVAL, "%s: temperature must be positive and finite", who);
+    if (sh->V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "%s: V=%d above 2^22", who, sh->V);
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaSetDevice");
+    return SPECDEC_OK;
+}
+}  // namespace
+
+int specdec_shard_stats(specdec_ctx* ctx, const specdec_shard* shard, const int32_t* cand_tokens,
+                        const int32_t* cand_len, float temperature, int B, int K, float* stats, void* stream) {
+    int rc = check_shard_args(ctx, shard, temperature, B, K, "shard_stats");
+    if (rc != SPECDEC_OK) return rc;
+    if (!cand_tokens || !stats) return fail(ctx, SPECDEC_EINVAL, "shard_stats: null pointer argument");
+    if (reinterpret_cast<uintptr_t>(stats) % 16 != 0) return fail(ctx, SPECDEC_EINVAL, "shard_stats: stats must be 16-byte aligned");
+    const float c = (float)(1.4426950408889634 / (double)temperature);
+    cudaError_t e = launch_shard_stats(*shard, cand_tokens, cand_len, c, B, K, stats, ctx->status, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "shard_stats launch");
+    ctx->launches += 1;
+    return SPECDEC_OK;
+}
+
+int specdec_shard_accept(specdec_ctx* ctx, const specdec_shard* shard, const float* stats_all, int n_shards,
+                         const int32_t* cand_len, const float* uniforms, float temperature, int B, int K,
+                         int32_t* n_accepted, float* accept_ratio, float* row_norm, double* mass, void* stream) {
+    int rc = check_shard_args(ctx, shard, temperature, B, K, "shard_accept");
+    if (rc != SPECDEC_OK) return rc;
+    if (!stats_all || !uniforms || !n_accepted || !row_norm || !mass) return fail(ctx, SPECDEC_EINVAL, "shard_accept: null pointer argument");
+    if (n_shards < 1 || n_shards > SPECDEC_SHARD_MAX_RANKS) return fail(ctx, SPECDEC_EINVAL, "shard_accept: n_shards must be in [1, %d] (got %d)", SPECDEC_SHARD_MAX_RANKS, n_shards);
+    if (reinterpret_cast<uintptr_t>(stats_all) % 16 != 0 || reinterpret_cast<uintptr_t>(row_norm) % 16 != 0)
+        return fail(ctx, SPECDEC_EINVAL, "shard_accept: stats_all and row_norm must be 16-byte aligned");
+    const float c = (float)(1.4426950408889634 / (double)temperature);
+    cudaError_t e = launch_shard_accept(*shard, stats_all, n_shards, cand_len, uniforms, c, B, K, n_accepted, accept_ratio,
+                                        row_norm, mass, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "shard_accept launch");
+    ctx->launches += 2;
+    return SPECDEC_OK;
+}
+
+int specdec_shard_draw(specdec_ctx* ctx, const specdec_shard* shard, const float* stats_all, const double* mass_all,
+                       int n_shards, int rank, const int32_t* n_accepted, const int32_t* cand_len,
+                       const float* uniforms, const float* row_norm, float temperature, int B, int K,
+                       int32_t* next_token, float* resid_mass, void* stream) {
+    int rc = check_shard_args(ctx, shard, temperature, B, K, "shard_draw");
+    if (rc != SPECDEC_OK) return rc;
+    if (!stats_all || !mass_all || !n_accepted || !uniforms || !row_norm || !next_token)
+        return fail(ctx, SPECDEC_EINVAL, "shard_draw: null pointer argument");
+    if (n_shards < 1 || n_shards > SPECDEC_SHARD_MAX_RANKS || rank < 0 || rank >= n_shards)
+        return fail(ctx, SPECDEC_EINVAL, "shard_draw: rank %d of %d shards (at most %d)", rank, n_shards, SPECDEC_SHARD_MAX_RANKS);
+    if (reinterpret_cast<uintptr_t>(stats_all) % 16 != 0 || reinterpret_cast<uintptr_t>(row_norm) % 16 != 0)
+        return fail(ctx, SPECDEC_EINVAL, "shard_draw: stats_all and row_norm must be 16-byte aligned");
+    const float c = (float)(1.4426950408889634 / (double)temperature);
+    cudaError_t e = launch_shard_draw(*shard, stats_all, mass_all, n_shards, rank, n_accepted, cand_len, uniforms, row_norm,
+                                      c, B, K, next_token, resid_mass, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "shard_draw launch");
+    ctx->launches += 1;
+    return SPECDEC_OK;
+}
+
 int specdec_verify_greedy(specdec_ctx* ctx, const void* target_logits, specdec_dtype dtype,
                           const int32_t* cand_tokens, const int32_t* cand_len, int B, int K, int V,
                           int32_t* n_accepted, int32_t* next_token, int32_t* target_argmax, void* stream) {

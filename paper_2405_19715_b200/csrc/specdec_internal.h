@@ -70,3 +70,12 @@ cudaError_t launch_stop_step(const float* accept_prob_step, float* p_hat, float 
                              cudaStream_t s);
 cudaError_t launch_wait_limit_selftest(uint32_t* status, cudaStream_t s);
 cudaError_t launch_verify_topk(const VerifyParams& p, specdec_dtype dtype, int top_k, cudaStream_t s);
+cudaError_t launch_shard_stats(const specdec_shard& sh, const int32_t* tokens, const int32_t* lens, float c, int B,
+                               int K, float* stats, uint32_t* status, cudaStream_t s);
+cudaError_t launch_shard_accept(const specdec_shard& sh, const float* stats_all, int n_shards, const int32_t* lens,
+                                const float* uniforms, float c, int B, int K, int32_t* n_acc, float* ratio,
+                                float* row_norm, double* mass, cudaStream_t s);
+cudaError_t launch_shard_draw(const specdec_shard& sh, const float* stats_all, const double* mass_all, int n_shards,
+                              int rank, const int32_t* n_acc, const int32_t* lens, const float* uniforms,
+                              const float* row_norm, float c, int B, int K, int32_t* next, float* rmass,
+                              cudaStream_t s);

@@ -53,59 +53,7 @@ __global__ void __launch_bounds__(DIRECT_THREADS, 2) verify_direct_kernel(const 
     // ---- pass 1: softmax statistics of both rows
     const int nvec = (P.V + N - 1) / N;
     Acc ap = acc_init(), aq = acc_init();
-    if constexpr (VEC) {
-        // four vectors of each row in flight per thread; the reference is moved from the maximum of
-        // the raw inputs, so the exponentials are issued without a data-dependent branch
-        constexpr int U = 4, NP = N / 2;
-        const uint4* tv = reinterpret_cast<const uint4*>(trow);
-        const uint4* dv = reinterpret_cast<const uint4*>(drow);
-        const uint32_t ninf = neg_inf_word(T());
-        Acc2 a2 = acc2_init(), q2 = acc2_init();
-        for (int j0 = tid; j0 < nvec; j0 += U * DIRECT_THREADS) {
-            uint4 rt[U], rd[U];
-#pragma unroll
-            for (int k = 0; k < U; ++k) {
-                const int j = j0 + k * DIRECT_THREADS;
-                rt[k] = rd[k] = make_uint4(ninf, ninf, ninf, ninf);
-                if (j < nvec) {
-                    rt[k] = __ldcg(tv + j);
-                    if (!u.bonus) rd[k] = __ldcg(dv + j);
-                }
-            }
-            float mt = -INFINITY, md = -INFINITY;
-#pragma unroll
-            for (int k = 0; k < U; ++k) {
-                mt = fmaxf(mt, vec_max(rt[k], T()));
-                md = fmaxf(md, vec_max(rd[k], T()));
-            }
-            acc2_reference_thread(a2, mt, P.c);
-            if (!u.bonus) acc2_reference_thread(q2, md, P.c);
-            const f2 c2 = pack2(P.c, P.c);
-            const f2 np2 = pack2(-a2.rs, -a2.rs), nq2 = pack2(-q2.rs, -q2.rs);
-#pragma unroll
-            for (int k = 0; k < U; ++k) {
-                f2 xt[NP], xd[NP];
-                to_pairs(rt[k], xt, T());
-                acc2_add<NP>(a2, xt, c2, np2);
-                if (!u.bonus) {
-                    to_pairs(rd[k], xd, T());
-                    acc2_add<NP>(q2, xd, c2, nq2);
-                }
-            }
-        }
-        ap = acc2_fold(a2);
-        aq = acc2_fold(q2);
-    } else {
-        float xt[N], xd[N];
-        for (int j = tid; j < nvec; j += DIRECT_THREADS) {
-            load_vec<T, VEC>(trow, j, P.V, xt);
-            acc_update<N>(ap, xt, P.c);
-            if (!u.bonus) {
-                load_vec<T, VEC>(drow, j, P.V, xd);
-                acc_update<N>(aq, xd, P.c);
-            }
-        }
-    }
+    unit_stats<T, VEC, DIRECT_THREADS>(trow, drow, P.V, P.c, u.bonus, tid, ap, aq);
     ap = warp_merge(ap);
     aq = warp_merge(aq);
     if (lane == 0) { sh.wp[warp] = ap; sh.wq[warp] = aq; }

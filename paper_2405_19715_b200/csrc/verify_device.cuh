@@ -262,6 +262,68 @@ __device__ __forceinline__ float prob(float x, float c, const Norm& n) {
     return ex2(fmaf(x, c, -n.hi) - n.lo);
 }
 
+// Pass over the two rows of one unit by a CTA of THREADS threads: this thread's share of the
+// softmax statistics (merge with warp_merge / acc_merge).  The draft row is skipped at a bonus
+// position.  VEC: four vectors of each row in flight per thread; the reference is moved from the
+// maximum of the raw inputs, so the exponentials are issued without a data-dependent branch.
+template <typename T, bool VEC, int THREADS>
+__device__ __forceinline__ void unit_stats(const T* __restrict__ trow, const T* __restrict__ drow, int V, float c,
+                                           bool bonus, int tid, Acc& ap, Acc& aq) {
+    constexpr int N = Elem<T>::EPV;
+    const int nvec = (V + N - 1) / N;
+    if constexpr (VEC) {
+        constexpr int U = 4, NP = N / 2;
+        const uint4* tv = reinterpret_cast<const uint4*>(trow);
+        const uint4* dv = reinterpret_cast<const uint4*>(drow);
+        const uint32_t ninf = neg_inf_word(T());
+        Acc2 a2 = acc2_init(), q2 = acc2_init();
+        for (int j0 = tid; j0 < nvec; j0 += U * THREADS) {
+            uint4 rt[U], rd[U];
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                const int j = j0 + k * THREADS;
+                rt[k] = rd[k] = make_uint4(ninf, ninf, ninf, ninf);
+                if (j < nvec) {
+                    rt[k] = __ldcg(tv + j);
+                    if (!bonus) rd[k] = __ldcg(dv + j);
+                }
+            }
+            float mt = -INFINITY, md = -INFINITY;
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                mt = fmaxf(mt, vec_max(rt[k], T()));
+                md = fmaxf(md, vec_max(rd[k], T()));
+            }
+            acc2_reference_thread(a2, mt, c);
+            if (!bonus) acc2_reference_thread(q2, md, c);
+            const f2 c2 = pack2(c, c);
+            const f2 np2 = pack2(-a2.rs, -a2.rs), nq2 = pack2(-q2.rs, -q2.rs);
+#pragma unroll
+            for (int k = 0; k < U; ++k) {
+                f2 xt[NP], xd[NP];
+                to_pairs(rt[k], xt, T());
+                acc2_add<NP>(a2, xt, c2, np2);
+                if (!bonus) {
+                    to_pairs(rd[k], xd, T());
+                    acc2_add<NP>(q2, xd, c2, nq2);
+                }
+            }
+        }
+        ap = acc2_fold(a2);
+        aq = acc2_fold(q2);
+    } else {
+        float xt[N], xd[N];
+        for (int j = tid; j < nvec; j += THREADS) {
+            load_vec<T, VEC>(trow, j, V, xt);
+            acc_update<N>(ap, xt, c);
+            if (!bonus) {
+                load_vec<T, VEC>(drow, j, V, xd);
+                acc_update<N>(aq, xd, c);
+            }
+        }
+    }
+}
+
 // Shared-memory scratch of one CTA handling one (row, position) unit.
 struct UnitShared {
     Acc wp[32], wq[32];        // per-warp partial statistics
@@ -353,7 +415,7 @@ template <typename T, bool VEC>
 __device__ __forceinline__ int draw_select(const VerifyParams& P, const T* __restrict__ trow,
                                            const T* __restrict__ drow, int mode, float u01, const Norm np,
                                            const Norm nq, const float* __restrict__ slab_sum, int lane,
-                                           double* total_out) {
+                                           double* total_out, double tau_abs = -1.0) {
     constexpr int N = Elem<T>::EPV;
     const int V = P.V;
     const int nvec = (V + N - 1) / N;
@@ -373,7 +435,8 @@ __device__ __forceinline__ int draw_select(const VerifyParams& P, const T* __res
         if (lane >= o) incl += up;
     }
     const double total = __shfl_sync(0xffffffffu, incl, 31);
-    const double tau = (double)u01 * total;
+    // the mass to walk to: u * total, unless the caller fixed it (a draw that spans several calls' rows)
+    const double tau = tau_abs >= 0.0 ? tau_abs : (double)u01 * total;
     // first slab whose inclusive prefix exceeds tau
     double run = incl - mine;
     int found = -1;
@@ -450,7 +513,8 @@ __device__ __forceinline__ int draw_select(const VerifyParams& P, const T* __res
 // named barrier `bar_id`.
 template <typename T, bool VEC>
 __device__ void unit_draw(const VerifyParams& P, const T* __restrict__ trow, const T* __restrict__ drow, int mode,
-                          float u01, UnitShared& sh, float* __restrict__ slab_sum, int tid, int nthreads, int bar_id) {
+                          float u01, UnitShared& sh, float* __restrict__ slab_sum, int tid, int nthreads, int bar_id,
+                          double tau_abs = -1.0) {
     constexpr int N = Elem<T>::EPV;
     const int V = P.V;
     const int nvec = (V + N - 1) / N;
@@ -510,7 +574,7 @@ __device__ void unit_draw(const VerifyParams& P, const T* __restrict__ trow, con
 
     if (warp == 0) {
         double total;
-        const int tok = draw_select<T, VEC>(P, trow, drow, mode, u01, np, nq, slab_sum, lane, &total);
+        const int tok = draw_select<T, VEC>(P, trow, drow, mode, u01, np, nq, slab_sum, lane, &total, tau_abs);
         if (lane == 0) { sh.token = tok; sh.total = total; }
     }
     bar_sync(bar_id, nthreads);

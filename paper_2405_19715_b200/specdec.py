@@ -19,7 +19,9 @@ DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT, DATA_TOPK_TIES = 1, 2, 4, 8
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
            "specdec_launch_count", "specdec_verify_correct", "specdec_verify_correct_host",
-           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step", "specdec_selftest_wait_limit", "specdec_verify_correct_topk", "specdec_sample"]
+           "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step", "specdec_selftest_wait_limit", "specdec_verify_correct_topk", "specdec_sample",
+           "specdec_shard_stats", "specdec_shard_accept", "specdec_shard_draw"]
+SHARD_STATS_WIDTH, SHARD_MAX_RANKS = 8, 64
 STATIC_MAX_UNITS, STATIC_MAX_V = 16384, 262144
 
 
@@ -32,6 +34,11 @@ class SpecdecError(RuntimeError):
 class _Head(C.Structure):
     _fields_ = [("W", C.POINTER(C.c_void_p)), ("b", C.POINTER(C.c_void_p)), ("w_out", C.c_void_p),
                 ("b_out", C.c_float), ("d", C.c_int), ("depth", C.c_int)]
+
+
+class _Shard(C.Structure):
+    _fields_ = [("target_logits", C.c_void_p), ("draft_logits", C.c_void_p), ("dtype", C.c_int),
+                ("V_shard", C.c_int), ("v_offset", C.c_int), ("V", C.c_int)]
 
 
 _lib = None
@@ -61,6 +68,12 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
     lib.specdec_verify_correct_topk.argtypes = [C.c_void_p, vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int, C.c_int,
                                                 C.c_int, C.c_int, ip, ip, fp, fp, C.c_void_p]
     lib.specdec_sample.argtypes = [C.c_void_p, vp, C.c_int, fp, C.c_float, C.c_int, C.c_int, C.c_int, ip, C.c_void_p]
+    sp = C.POINTER(_Shard)
+    lib.specdec_shard_stats.argtypes = [C.c_void_p, sp, ip, ip, C.c_float, C.c_int, C.c_int, fp, C.c_void_p]
+    lib.specdec_shard_accept.argtypes = [C.c_void_p, sp, fp, C.c_int, ip, fp, C.c_float, C.c_int, C.c_int, ip, fp, fp,
+                                         vp, C.c_void_p]
+    lib.specdec_shard_draw.argtypes = [C.c_void_p, sp, fp, vp, C.c_int, C.c_int, ip, ip, fp, fp, C.c_float, C.c_int,
+                                       C.c_int, ip, fp, C.c_void_p]
     lib.specdec_selftest_wait_limit.argtypes = [C.c_void_p, C.c_void_p]
     lib.specdec_stop_step.argtypes = [C.c_void_p, fp, fp, C.c_float, C.c_int, ip, C.c_void_p]
     lib.specdec_verify_greedy.argtypes = [C.c_void_p, vp, C.c_int, ip, ip, C.c_int, C.c_int, C.c_int, ip, ip, ip,
@@ -221,6 +234,58 @@ def specdec_sample(ctx: Context, logits, uniforms, temperature: float, top_k: in
                                 float(temperature), int(top_k), B, V, _ptr(tokens, torch.int32), _stream(stream))
     ctx._check(rc)
     return tokens
+
+
+def _shard(target_shard, draft_shard, v_offset: int, V: int) -> _Shard:
+    return _Shard(_ptr(target_shard), _ptr(draft_shard), _logit_dtype(target_shard), target_shard.shape[2],
+                  int(v_offset), int(V))
+
+
+def specdec_shard_stats(ctx: Context, target_shard, draft_shard, v_offset: int, V: int, cand_tokens, cand_len,
+                        temperature: float, stats=None, stream=None):
+    """specdec_shard_stats of the C ABI.  Returns stats [B, K+1, 8] fp32 (device)."""
+    B, K1, _ = target_shard.shape
+    if stats is None:
+        stats = torch.empty(B, K1, SHARD_STATS_WIDTH, dtype=torch.float32, device=target_shard.device)
+    sh = _shard(target_shard, draft_shard, v_offset, V)
+    rc = ctx.lib.specdec_shard_stats(ctx.handle, C.byref(sh), _ptr(cand_tokens, torch.int32),
+                                     _ptr(cand_len, torch.int32), float(temperature), B, K1 - 1,
+                                     _ptr(stats, torch.float32), _stream(stream))
+    ctx._check(rc)
+    return stats
+
+
+def specdec_shard_accept(ctx: Context, target_shard, draft_shard, v_offset: int, V: int, stats_all, cand_len,
+                         uniforms, temperature: float, accept_ratio=None, stream=None):
+    """specdec_shard_accept of the C ABI.  Returns (n_accepted [B] int32, row_norm [B, 4] fp32, mass [B] fp64)."""
+    B, K1, _ = target_shard.shape
+    dev = target_shard.device
+    n_accepted = torch.empty(B, dtype=torch.int32, device=dev)
+    row_norm = torch.empty(B, 4, dtype=torch.float32, device=dev)
+    mass = torch.empty(B, dtype=torch.float64, device=dev)
+    sh = _shard(target_shard, draft_shard, v_offset, V)
+    rc = ctx.lib.specdec_shard_accept(ctx.handle, C.byref(sh), _ptr(stats_all, torch.float32), stats_all.shape[0],
+                                      _ptr(cand_len, torch.int32), _ptr(uniforms, torch.float32), float(temperature),
+                                      B, K1 - 1, _ptr(n_accepted, torch.int32), _ptr(accept_ratio, torch.float32),
+                                      _ptr(row_norm, torch.float32), _ptr(mass, torch.float64), _stream(stream))
+    ctx._check(rc)
+    return n_accepted, row_norm, mass
+
+
+def specdec_shard_draw(ctx: Context, target_shard, draft_shard, v_offset: int, V: int, stats_all, mass_all, rank: int,
+                       n_accepted, cand_len, uniforms, row_norm, temperature: float, resid_mass=None, stream=None):
+    """specdec_shard_draw of the C ABI.  Returns next_token [B] int32, -1 where another rank draws."""
+    B, K1, _ = target_shard.shape
+    next_token = torch.empty(B, dtype=torch.int32, device=target_shard.device)
+    sh = _shard(target_shard, draft_shard, v_offset, V)
+    rc = ctx.lib.specdec_shard_draw(ctx.handle, C.byref(sh), _ptr(stats_all, torch.float32),
+                                    _ptr(mass_all, torch.float64), stats_all.shape[0], int(rank),
+                                    _ptr(n_accepted, torch.int32), _ptr(cand_len, torch.int32),
+                                    _ptr(uniforms, torch.float32), _ptr(row_norm, torch.float32), float(temperature),
+                                    B, K1 - 1, _ptr(next_token, torch.int32), _ptr(resid_mass, torch.float32),
+                                    _stream(stream))
+    ctx._check(rc)
+    return next_token
 
 
 def specdec_selftest_wait_limit(ctx: Context, stream=None):
