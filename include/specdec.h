@@ -132,7 +132,7 @@ int specdec_verify_correct(specdec_ctx* ctx,
  * exactly as in specdec_verify_correct.  A drafted token outside the target's kept set is rejected
  * with certainty; y' always lies in the target's kept set.  top_k >= V is the unfiltered
  * operation.  Arguments as for specdec_verify_correct; 1 <= top_k <= 256 (or >= V).
- * The kept logits' probabilities are evaluated in fp64.  Logits equal to the k-th largest are all
+ * The kept logits are evaluated like the unfiltered ones (fp32 terms, fp64 prefix sums).  Logits equal to the k-th largest are all
  * kept.  Where more than 2048 logits of a target row, or 4096 of a draft row, are kept that way the
  * call sets SPECDEC_DATA_TOPK_TIES: an accept test it touches reports n_accepted = -1, a draw it
  * touches next_token = -1.

@@ -3,18 +3,21 @@
 // runs on the filtered distributions.
 //
 // Only about k logits per row matter, so nothing is exponentiated while streaming.  One CTA per
-// (row, position), two passes per logit row:
-//   1. every thread takes the maximum of its strided share of the row; the smallest, over warps, of
-//      each warp's r-th largest thread maximum (r = ceil(k / warps)) is a lower bound on the k-th
-//      largest of the row, and a tight one: a thread's share holds 1/512 of the row, so few of the
-//      top k collide in one share;
-//   2. the row is read again, newest lines first so that they still sit in L2, and every logit at or
-//      above the bound goes into a candidate buffer in shared memory (k plus a few tens).
-// The exact k-th largest is found among the candidates (rank counting, radix select when there are
-// many), and the softmax terms, the accept test and -- for a rejecting or bonus position -- the
-// residual draw are evaluated on the kept candidates in fp64 by the whole CTA.  If the bound turns
-// out too loose for the buffer (rows with -inf or repeated maxima), an exact radix select over the
-// row supplies the threshold and the row is filtered again.
+// (row, position); per logit row:
+//   1. every thread takes the maximum of its strided share of the row (the one pass that comes
+//      from HBM); the smallest, over warps, of each warp's r-th largest thread maximum
+//      (r = ceil(k / warps)) is a lower bound on the k-th largest of the row, and a tight one: a
+//      share holds 1/512 of the row, so few of the top k collide in one share;
+//   2. the shares whose maximum reached the bound (about k of 512) are read again, from L2, a warp
+//      per share, and every logit at or above the bound goes into a candidate buffer in shared
+//      memory (k plus a few tens);
+//   3. the exact k-th largest of the candidates is built bit by bit from counting barriers (each
+//      thread holds up to two candidates' order-preserving keys; a radix select takes over when
+//      there are more), and the softmax terms of the kept ones are summed.
+// The accept test follows, and -- for a rejecting or bonus position -- the residual draw over the
+// kept entries: ranked by token id, weights in fp32, prefix in fp64 (the arithmetic of the
+// unfiltered kernels).  If the bound turns out too loose for the buffer (rows with -inf or repeated
+// maxima), an exact radix select over the row supplies the threshold and the row is filtered again.
 #include "verify_device.cuh"
 
 namespace {
@@ -25,17 +28,19 @@ constexpr int TK_THREADS = 512;
 constexpr int TK_WARPS = TK_THREADS / 32;
 constexpr int CAP = 4096;                 // candidates per row; every V <= CAP fits whole
 constexpr int MAX_KEPT = CAP / 2;         // kept entries (k + ties at the k-th value) the draw can hold
-constexpr int RANK_COUNT_MAX = 1024;      // above this many candidates the k-th largest comes from a radix select
+constexpr int FB = 4;                     // flagged shares a warp reads per trip
 
 struct TkShared {
-    float warp_rth[2][TK_WARPS];
-    float bound[2], tau[2];
+    float wrth[TK_WARPS], wmax[TK_WARPS];
+    long long zpart[TK_WARPS];
     int count[2], overflow[2];
+    float tau[2];
+    Norm norm[2];
     unsigned int hist[256];
     unsigned int sel_prefix, sel_rank;
-    double zsum[2], dmax[2];
-    int state, n_kept, token, retry;
+    int state, n_kept, token, retry, nflag;
     float mass;
+    unsigned short flist[TK_THREADS];              // threads whose share holds a candidate
 };
 
 __device__ __forceinline__ uint32_t order_key(float x) {        // larger float <-> larger key; NaN sorts lowest
@@ -91,49 +96,67 @@ __device__ __forceinline__ float thread_max(const T* __restrict__ row, int V, in
     return m;
 }
 
-// Pass 2: every logit at or above the bound goes into the candidate buffer, last lines first.
+__device__ __forceinline__ void append(float x, int idx, float* cval, int* cidx, int* count, int* overflow) {
+    const int pos = atomicAdd(count, 1);
+    if (pos < CAP) { cval[pos] = x; cidx[pos] = idx; }
+    else *overflow = 1;
+}
+
+// Pass 2: every logit at or above the bound goes into the candidate buffer.  Only the shares whose
+// maximum reached the bound are read again (from L2): a share is the strided set of vectors one
+// thread covered in pass 1; a warp takes FB such shares per trip, one vector per lane and share.
 template <typename T, bool VEC>
-__device__ __forceinline__ void filter_row(const T* __restrict__ row, int V, float bound, float* cval, int* cidx,
-                                           int* count, int* overflow, int tid) {
+__device__ __forceinline__ void filter_row(const T* __restrict__ row, int V, float bound, float my_max, float* cval,
+                                           int* cidx, int* count, int* overflow, TkShared& sh, int tid) {
     constexpr int N = Elem<T>::EPV;
+    const int lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) sh.nflag = 0;
+    __syncthreads();
+    if (my_max >= bound) sh.flist[atomicAdd(&sh.nflag, 1)] = (unsigned short)tid;
+    __syncthreads();
+    const int nflag = sh.nflag;
     if constexpr (VEC) {
-        constexpr int U = 4;
-        constexpr int STEP = U * TK_THREADS;
         const int nvec = V / N;
         const uint4* rv = reinterpret_cast<const uint4*>(row);
-        const uint32_t ninf = neg_inf_word(T());
-        for (int base = ((nvec - 1) / STEP) * STEP; base >= 0; base -= STEP) {
-            uint4 r[U];
+        for (int f0 = warp; f0 < nflag; f0 += TK_WARPS * FB) {
+            uint4 r[FB];
+            int jj[FB];
 #pragma unroll
-            for (int k = 0; k < U; ++k) {
-                const int j = base + tid + k * TK_THREADS;
-                r[k] = j < nvec ? __ldcg(rv + j) : make_uint4(ninf, ninf, ninf, ninf);
+            for (int q = 0; q < FB; ++q) {
+                const int f = f0 + q * TK_WARPS;
+                jj[q] = f < nflag ? (int)sh.flist[f] + TK_THREADS * lane : nvec;
+                if (jj[q] < nvec) r[q] = __ldcg(rv + jj[q]);
             }
 #pragma unroll
-            for (int k = 0; k < U; ++k) {
-                const int j = base + tid + k * TK_THREADS;
-                if (j < nvec && vec_max(r[k], T()) >= bound) {
+            for (int q = 0; q < FB; ++q) {
+                if (jj[q] < nvec && vec_max(r[q], T()) >= bound) {
                     float x[N];
-                    unpack(r[k], x);
+                    unpack(r[q], x);
 #pragma unroll
                     for (int e = 0; e < N; ++e)
-                        if (x[e] >= bound) {
-                            const int pos = atomicAdd(count, 1);
-                            if (pos < CAP) { cval[pos] = x[e]; cidx[pos] = j * N + e; }
-                            else *overflow = 1;
-                        }
+                        if (x[e] >= bound) append(x[e], jj[q] * N + e, cval, cidx, count, overflow);
                 }
             }
         }
-    } else {
-        for (int v = tid; v < V; v += TK_THREADS) {
-            const float x = to_float(row[v]);
-            if (x >= bound) {
-                const int pos = atomicAdd(count, 1);
-                if (pos < CAP) { cval[pos] = x; cidx[pos] = v; }
-                else *overflow = 1;
-            }
+        if (nvec > TK_THREADS * 32) {                  // rows longer than one vector per lane and share
+            for (int f = warp; f < nflag; f += TK_WARPS)
+                for (int j = (int)sh.flist[f] + TK_THREADS * (lane + 32); j < nvec; j += TK_THREADS * 32) {
+                    const uint4 r = __ldcg(rv + j);
+                    if (vec_max(r, T()) >= bound) {
+                        float x[N];
+                        unpack(r, x);
+#pragma unroll
+                        for (int e = 0; e < N; ++e)
+                            if (x[e] >= bound) append(x[e], j * N + e, cval, cidx, count, overflow);
+                    }
+                }
         }
+    } else {
+        for (int f = warp; f < nflag; f += TK_WARPS)
+            for (int v = (int)sh.flist[f] + TK_THREADS * lane; v < V; v += TK_THREADS * 32) {
+                const float x = to_float(row[v]);
+                if (x >= bound) append(x, v, cval, cidx, count, overflow);
+            }
     }
 }
 
@@ -188,6 +211,32 @@ __device__ float radix_kth_largest(F at, int n, int k, TkShared& sh, int tid) {
     return key_to_float(prefix);
 }
 
+// Exact k-th largest of n <= 2 * TK_THREADS values in shared memory: the key is built from the top
+// bit down, each bit decided by one counting barrier ("are there still k keys at or above this?").
+// bf16 data needs only the upper half of the key.  Every thread calls it and gets the result.
+template <typename T>
+__device__ __forceinline__ float bisect_kth_largest(const float* cv, int n, int k, int tid) {
+    const bool h0 = tid < n, h1 = tid + TK_THREADS < n;
+    const uint32_t k0 = h0 ? order_key(cv[tid]) : 0u, k1 = h1 ? order_key(cv[tid + TK_THREADS]) : 0u;
+    constexpr int LOW = sizeof(T) == 2 ? 16 : 0;
+    uint32_t prefix = 0;
+    if (n <= TK_THREADS) {
+        for (int bit = 31; bit >= LOW; --bit) {
+            const uint32_t t = prefix | (1u << bit);
+            if (__syncthreads_count(h0 && k0 >= t) >= k) prefix = t;
+        }
+    } else {
+        for (int bit = 31; bit >= LOW; --bit) {
+            const uint32_t t = prefix | (1u << bit);
+            const int c = __syncthreads_count(h0 && k0 >= t) + __syncthreads_count(h1 && k1 >= t);
+            if (c >= k) prefix = t;
+        }
+    }
+    // the low half of a widened bf16's key is all zeros (positive) or all ones (negative)
+    if (LOW && !(prefix & 0x80000000u)) prefix |= 0xffffu;
+    return key_to_float(prefix);
+}
+
 template <typename T, bool VEC>
 __global__ void __launch_bounds__(TK_THREADS, 2) verify_topk_kernel(const VerifyParams P, int top_k) {
     extern __shared__ __align__(16) unsigned char tk_smem[];
@@ -218,6 +267,7 @@ __global__ void __launch_bounds__(TK_THREADS, 2) verify_topk_kernel(const Verify
     rows[1] = u.bonus ? rows[0] : static_cast<const T*>(P.draft) + ((size_t)u.b * P.K + u.i) * (size_t)V;
     const int nrows = u.bonus ? 1 : 2;
     const int k = min(top_k, V);
+    const float c = P.c;
 
     // accept-test operands, requested early
     int y = 0, y_ok = 1;
@@ -232,82 +282,73 @@ __global__ void __launch_bounds__(TK_THREADS, 2) verify_topk_kernel(const Verify
 
     const int rth = (k + TK_WARPS - 1) / TK_WARPS;
     for (int rr = 0; rr < nrows; ++rr) {
-        // ---- pass 1: a lower bound on the k-th largest of the row
-        const float wr = warp_rth_largest(thread_max<T, VEC>(rows[rr], V, tid), rth, lane);
-        if (lane == 0) sh.warp_rth[rr][warp] = wr;
+        // ---- pass 1: the row's maximum and a lower bound on its k-th largest
+        const float my_max = thread_max<T, VEC>(rows[rr], V, tid);
+        const float wr = warp_rth_largest(my_max, rth, lane);
+        float wm;
+        asm("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(wm) : "f"(my_max));
+        if (lane == 0) { sh.wrth[warp] = wr; sh.wmax[warp] = wm; }
         __syncthreads();
-        float b = sh.warp_rth[rr][0];
+        float bound = sh.wrth[0], row_max = sh.wmax[0];
 #pragma unroll
-        for (int w = 1; w < TK_WARPS; ++w) b = fminf(b, sh.warp_rth[rr][w]);
+        for (int w = 1; w < TK_WARPS; ++w) { bound = fminf(bound, sh.wrth[w]); row_max = fmaxf(row_max, sh.wmax[w]); }
         // ---- pass 2: candidates at or above the bound
         float* cv = cval + rr * CAP;
         int* ci = cidx + rr * CAP;
-        filter_row<T, VEC>(rows[rr], V, b, cv, ci, &sh.count[rr], &sh.overflow[rr], tid);
+        filter_row<T, VEC>(rows[rr], V, bound, my_max, cv, ci, &sh.count[rr], &sh.overflow[rr], sh, tid);
         __syncthreads();
         if (sh.overflow[rr]) {                         // block-uniform: the bound was too loose
             const T* row = rows[rr];
             const float kth = radix_kth_largest([row](int v) { return to_float(row[v]); }, V, k, sh, tid);
             if (tid == 0) { sh.count[rr] = 0; sh.overflow[rr] = 0; }
             __syncthreads();
-            filter_row<T, VEC>(row, V, kth, cv, ci, &sh.count[rr], &sh.overflow[rr], tid);
+            filter_row<T, VEC>(row, V, kth, my_max, cv, ci, &sh.count[rr], &sh.overflow[rr], sh, tid);
             __syncthreads();
         }
 
-        // ---- exact k-th largest among the candidates, softmax terms of the kept ones (fp64)
+        // ---- exact k-th largest among the candidates; n <= k: all are kept, tau is their minimum
         const int n = min(sh.count[rr], CAP);
-        const int kk = min(k, n);                      // n <= k: every candidate is kept, tau is their minimum
+        const int kk = min(k, n);
         float tau = -INFINITY;
-        if (n > RANK_COUNT_MAX) {
-            tau = radix_kth_largest([cv](int c) { return cv[c]; }, n, kk, sh, tid);
-        } else if (n > 0) {
-            if (tid == 0) sh.tau[rr] = -INFINITY;
-            __syncthreads();
-            for (int c = tid; c < n; c += TK_THREADS) {
-                const float vc = cv[c];
-                int gt = 0, ge = 0;
-                for (int j = 0; j < n; ++j) { gt += cv[j] > vc; ge += cv[j] >= vc; }
-                if (gt < kk && kk <= ge) sh.tau[rr] = vc;             // every such c carries the same value
-            }
-            __syncthreads();
-            tau = sh.tau[rr];
-        }
-        float m = -INFINITY;
-        for (int c = tid; c < n; c += TK_THREADS) if (cv[c] >= tau) m = fmaxf(m, cv[c]);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-        if (lane == 0) sh.warp_rth[rr][warp] = m;
-        if (tid == 0) { sh.tau[rr] = tau; sh.zsum[rr] = 0.0; }
-        __syncthreads();
-        float mm = sh.warp_rth[rr][0];
-#pragma unroll
-        for (int w = 1; w < TK_WARPS; ++w) mm = fmaxf(mm, sh.warp_rth[rr][w]);
-        const double dm = (double)mm, cc = (double)P.c;
-        double z = 0.0;
-        for (int c = tid; c < n; c += TK_THREADS) if (cv[c] >= tau) z += exp2(((double)cv[c] - dm) * cc);
+        if (n > 2 * TK_THREADS) tau = radix_kth_largest([cv](int q) { return cv[q]; }, n, kk, sh, tid);
+        else if (n > 0) tau = bisect_kth_largest<T>(cv, n, kk, tid);
+
+        // ---- softmax terms of the kept candidates against the row maximum (always kept), summed in
+        //      fixed point: the candidates sit in the buffer in arrival order, and integer addition
+        //      makes the sum independent of it
+        const float ref = row_max * c;
+        long long z = 0;
+        for (int q = tid; q < n; q += TK_THREADS)
+            if (cv[q] >= tau) z += (long long)(ex2(fmaf(cv[q], c, -ref)) * 1099511627776.f);       // 2^40
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
-        if (lane == 0 && z != 0.0) atomicAdd(&sh.zsum[rr], z);
-        if (tid == 0) sh.dmax[rr] = dm;
+        if (lane == 0) sh.zpart[warp] = z;
         __syncthreads();
+        if (tid == 0) {
+            long long zt = 0;
+            for (int w = 0; w < TK_WARPS; ++w) zt += sh.zpart[w];
+            const float zs = (float)((double)zt * (1.0 / 1099511627776.0));
+            sh.norm[rr] = make_norm(Acc{ref, zs});
+            sh.tau[rr] = tau;
+        }
     }
+    __syncthreads();
     const bool too_many_ties = sh.overflow[0] || (nrows == 2 && sh.overflow[1]);
 
     // ---- accept test (thread 0)
-    const double cc = (double)P.c;
     const float tau_p = sh.tau[0], tau_q = nrows == 2 ? sh.tau[1] : -INFINITY;
-    const double mp = sh.dmax[0], zp = sh.zsum[0];
-    const double mq = nrows == 2 ? sh.dmax[1] : 0.0, zq = nrows == 2 ? sh.zsum[1] : 1.0;
+    const Norm np = sh.norm[0], nq = nrows == 2 ? sh.norm[1] : sh.norm[0];
     if (tid == 0) {
         int state = 0;
         if (!u.bonus) {
-            double ratio;
+            float ratio;
             const bool p_in = y_ok && t_y >= tau_p && t_y > -INFINITY, q_in = y_ok && d_y >= tau_q && d_y > -INFINITY;
-            if (!p_in) ratio = 0.0;                                      // p'(y) = 0: certain rejection
+            if (!p_in) ratio = 0.f;                                      // p'(y) = 0: certain rejection
             else if (!q_in) ratio = INFINITY;
-            else ratio = exp2((((double)t_y - mp) - ((double)d_y - mq)) * cc) * (zq / zp);
-            state = (!y_ok || too_many_ties) ? FLAG_BAD : ((double)r_acc >= ratio ? FLAG_REJECT : FLAG_ACCEPT);
+            else ratio = exp2f((fmaf(t_y, c, -np.hi) - np.lo) - (fmaf(d_y, c, -nq.hi) - nq.lo));
+            state = (!y_ok || too_many_ties) ? FLAG_BAD : (r_acc >= ratio ? FLAG_REJECT : FLAG_ACCEPT);
             if (!y_ok) atomicOr(P.status, SPECDEC_DATA_BAD_TOKEN);
-            if (P.ratio) P.ratio[(size_t)u.b * P.K + u.i] = state == FLAG_BAD ? -1.f : (float)fmin(1.0, ratio);
+            if (P.ratio) P.ratio[(size_t)u.b * P.K + u.i] = state == FLAG_BAD ? -1.f : fminf(1.f, ratio);
             st_relaxed(&P.flags[(size_t)u.b * P.K + u.i], (int)((P.epoch << 2) | (uint32_t)state));
         }
         if (too_many_ties) atomicOr(P.status, SPECDEC_DATA_TOPK_TIES);
@@ -327,41 +368,47 @@ __global__ void __launch_bounds__(TK_THREADS, 2) verify_topk_kernel(const Verify
         const int n = min(sh.count[0], CAP);
         int* ki = cidx + CAP;                          // the draft row's buffers are free to reuse now
         float* kv = cval + CAP;
-        for (int c = tid; c < n; c += TK_THREADS)
-            if (cval[c] >= tau_p) {
+        for (int q = tid; q < n; q += TK_THREADS)
+            if (cval[q] >= tau_p) {
                 const int pos = atomicAdd(&sh.n_kept, 1);
-                if (pos < MAX_KEPT) { ki[pos] = cidx[c]; kv[pos] = cval[c]; }
+                if (pos < MAX_KEPT) { ki[pos] = cidx[q]; kv[pos] = cval[q]; }
             }
         __syncthreads();
         const int kept = sh.n_kept;
         if (kept > MAX_KEPT) {                         // thousands of ties at the k-th value
             if (tid == 0) atomicOr(P.status, SPECDEC_DATA_TOPK_TIES);
         } else {
-            int* si = cidx;                            // sorted indices; the target's candidates are consumed
-            double* sw = reinterpret_cast<double*>(cval);      // [MAX_KEPT] weights in vocabulary order
+            int* si = cidx;                            // token ids in vocabulary order; the target's candidates are consumed
+            int* kr = cidx + CAP / 2;                  // rank of each kept entry
+            float* sw = cval;                          // weights in vocabulary order
             const T* drow = rows[1];
+            for (int a = warp; a < kept; a += TK_WARPS) {      // position of entry a in vocabulary order
+                const int ia = ki[a];
+                int rank = 0;
+                for (int j = lane; j < kept; j += 32) rank += ki[j] < ia;
+                rank = __reduce_add_sync(0xffffffffu, rank);
+                if (lane == 0) kr[a] = rank;
+            }
             for (int pass = 0; pass < 2; ++pass) {
                 const bool resid = !u.bonus && pass == 0;
                 __syncthreads();
                 for (int a = tid; a < kept; a += TK_THREADS) {
                     const int ia = ki[a];
-                    int rank = 0;
-                    for (int j = 0; j < kept; ++j) rank += ki[j] < ia;
-                    double w = exp2(((double)kv[a] - mp) * cc) / zp;
+                    float w = prob(kv[a], c, np);
                     if (resid) {
                         const float dv = to_float(drow[ia]);
-                        const double qv = (dv >= tau_q && dv > -INFINITY) ? exp2(((double)dv - mq) * cc) / zq : 0.0;
-                        w = fmax(w - qv, 0.0);
+                        const float qv = (dv >= tau_q && dv > -INFINITY) ? prob(dv, c, nq) : 0.f;
+                        w = fmaxf(w - qv, 0.f);
                     }
-                    si[rank] = ia;
-                    sw[rank] = w;
+                    si[kr[a]] = ia;
+                    sw[kr[a]] = w;
                 }
                 __syncthreads();
                 if (warp == 0) {
                     // lane l sums entries [l*seg, (l+1)*seg); a warp scan gives the mass before each segment
                     const int seg = (kept + 31) / 32, a0 = min(lane * seg, kept), a1 = min(a0 + seg, kept);
                     double own = 0.0;
-                    for (int a = a0; a < a1; ++a) own += sw[a];
+                    for (int a = a0; a < a1; ++a) own += (double)sw[a];
                     double incl = own;
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) {
@@ -374,13 +421,13 @@ __global__ void __launch_bounds__(TK_THREADS, 2) verify_topk_kernel(const Verify
                         const double thr = (double)P.uniforms[(size_t)u.b * (P.K + 1) + P.K] * tot;
                         const unsigned hit = __ballot_sync(0xffffffffu, incl > thr);
                         int lastpos = -1;
-                        for (int a = a0; a < a1; ++a) if (sw[a] > 0.0) lastpos = a;
+                        for (int a = a0; a < a1; ++a) if (sw[a] > 0.f) lastpos = a;
                         if (hit) {
                             if (lane == __ffs(hit) - 1) {
                                 double run = incl - own;
                                 int tok = -1;
                                 for (int a = a0; a < a1; ++a) {
-                                    run += sw[a];
+                                    run += (double)sw[a];
                                     if (run > thr) { tok = si[a]; break; }
                                 }
                                 if (tok < 0 && lastpos >= 0) tok = si[lastpos];   // rounding at the segment's end
