@@ -8,9 +8,9 @@
 //      from HBM); the smallest, over warps, of each warp's r-th largest thread maximum
 //      (r = ceil(k / warps)) is a lower bound on the k-th largest of the row, and a tight one: a
 //      share holds 1/512 of the row, so few of the top k collide in one share;
-//   2. the shares whose maximum reached the bound (about k of 512) are read again, from L2, a warp
-//      per share, and every logit at or above the bound goes into a candidate buffer in shared
-//      memory (k plus a few tens);
+//   2. the pieces of shares (an eighth each) whose maximum reached the bound, about k of 4096, are
+//      read again, from L2, and every logit at or above the bound goes into a candidate buffer in
+//      shared memory (k plus a few tens);
 //   3. the exact k-th largest of the candidates is built bit by bit from counting barriers (each
 //      thread holds up to two candidates' order-preserving keys; a radix select takes over when
 //      there are more), and the softmax terms of the kept ones are summed.
@@ -28,7 +28,6 @@ constexpr int TK_THREADS = 512;
 constexpr int TK_WARPS = TK_THREADS / 32;
 constexpr int CAP = 4096;                 // candidates per row; every V <= CAP fits whole
 constexpr int MAX_KEPT = CAP / 2;         // kept entries (k + ties at the k-th value) the draw can hold
-constexpr int FB = 4;                     // flagged shares a warp reads per trip
 
 struct TkShared {
     float wrth[TK_WARPS], wmax[TK_WARPS];
@@ -40,7 +39,7 @@ struct TkShared {
     unsigned int sel_prefix, sel_rank;
     int state, n_kept, token, retry, nflag;
     float mass;
-    unsigned short flist[TK_THREADS];              // threads whose share holds a candidate
+    unsigned short flist[TK_THREADS * 8];          // (thread, sub-share) pairs that hold a candidate
 };
 
 __device__ __forceinline__ uint32_t order_key(float x) {        // larger float <-> larger key; NaN sorts lowest
@@ -67,32 +66,44 @@ __device__ __forceinline__ float warp_rth_largest(float v, int r, int lane) {
     return cur;
 }
 
-// Pass 1: this thread's maximum over its strided share of the row (NaN ignored).
+// Pass 1: this thread's maxima over its strided share of the row (NaN ignored).  The share is the
+// vectors tid + 512 q; it is kept as SEG sub-shares (q / U mod SEG) so that pass 2 can re-read a
+// few vectors instead of the whole share.  Without vector loads the share is one piece (seg[0]).
+constexpr int SEG = 8, TM_U = 4;
 template <typename T, bool VEC>
-__device__ __forceinline__ float thread_max(const T* __restrict__ row, int V, int tid) {
+__device__ __forceinline__ float thread_max(const T* __restrict__ row, int V, int tid, float (&seg)[SEG]) {
     constexpr int N = Elem<T>::EPV;
-    float m = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < SEG; ++s) seg[s] = -INFINITY;
     if constexpr (VEC) {
-        constexpr int U = 4;
         const int nvec = V / N;
         const uint4* rv = reinterpret_cast<const uint4*>(row);
         const uint32_t ninf = neg_inf_word(T());
-        for (int j0 = tid; j0 < nvec; j0 += U * TK_THREADS) {
-            uint4 r[U];
+        for (int base = 0; base < nvec; base += SEG * TM_U * TK_THREADS) {
 #pragma unroll
-            for (int k = 0; k < U; ++k) {
-                const int j = j0 + k * TK_THREADS;
-                r[k] = j < nvec ? __ldcg(rv + j) : make_uint4(ninf, ninf, ninf, ninf);
+            for (int s = 0; s < SEG; ++s) {
+                const int j0 = base + s * TM_U * TK_THREADS + tid;
+                if (j0 < nvec) {
+                    uint4 r[TM_U];
+#pragma unroll
+                    for (int k = 0; k < TM_U; ++k) {
+                        const int j = j0 + k * TK_THREADS;
+                        r[k] = j < nvec ? __ldcg(rv + j) : make_uint4(ninf, ninf, ninf, ninf);
+                    }
+#pragma unroll
+                    for (int k = 0; k < TM_U; ++k) seg[s] = fmaxf(seg[s], vec_max(r[k], T()));
+                }
             }
-#pragma unroll
-            for (int k = 0; k < U; ++k) m = fmaxf(m, vec_max(r[k], T()));
         }
     } else {
         for (int v = tid; v < V; v += TK_THREADS) {
             const float x = to_float(row[v]);
-            if (x == x) m = fmaxf(m, x);
+            if (x == x) seg[0] = fmaxf(seg[0], x);
         }
     }
+    float m = seg[0];
+#pragma unroll
+    for (int s = 1; s < SEG; ++s) m = fmaxf(m, seg[s]);
     return m;
 }
 
@@ -102,58 +113,44 @@ __device__ __forceinline__ void append(float x, int idx, float* cval, int* cidx,
     else *overflow = 1;
 }
 
-// Pass 2: every logit at or above the bound goes into the candidate buffer.  Only the shares whose
-// maximum reached the bound are read again (from L2): a share is the strided set of vectors one
-// thread covered in pass 1; a warp takes FB such shares per trip, one vector per lane and share.
+// Pass 2: every logit at or above the bound goes into the candidate buffer.  Only the sub-shares
+// whose maximum reached the bound are read again (from L2): four lanes per flagged sub-share, one
+// vector each.
 template <typename T, bool VEC>
-__device__ __forceinline__ void filter_row(const T* __restrict__ row, int V, float bound, float my_max, float* cval,
-                                           int* cidx, int* count, int* overflow, TkShared& sh, int tid) {
+__device__ __forceinline__ void filter_row(const T* __restrict__ row, int V, float bound, const float (&seg)[SEG],
+                                           float* cval, int* cidx, int* count, int* overflow, TkShared& sh, int tid) {
     constexpr int N = Elem<T>::EPV;
     const int lane = tid & 31, warp = tid >> 5;
     if (tid == 0) sh.nflag = 0;
     __syncthreads();
-    if (my_max >= bound) sh.flist[atomicAdd(&sh.nflag, 1)] = (unsigned short)tid;
+#pragma unroll
+    for (int s = 0; s < (VEC ? SEG : 1); ++s)
+        if (seg[s] >= bound) sh.flist[atomicAdd(&sh.nflag, 1)] = (unsigned short)(tid | (s << 9));
     __syncthreads();
     const int nflag = sh.nflag;
     if constexpr (VEC) {
+        static_assert(TM_U == 4 && TK_THREADS == 512, "entry packing and lane mapping");
         const int nvec = V / N;
         const uint4* rv = reinterpret_cast<const uint4*>(row);
-        for (int f0 = warp; f0 < nflag; f0 += TK_WARPS * FB) {
-            uint4 r[FB];
-            int jj[FB];
-#pragma unroll
-            for (int q = 0; q < FB; ++q) {
-                const int f = f0 + q * TK_WARPS;
-                jj[q] = f < nflag ? (int)sh.flist[f] + TK_THREADS * lane : nvec;
-                if (jj[q] < nvec) r[q] = __ldcg(rv + jj[q]);
-            }
-#pragma unroll
-            for (int q = 0; q < FB; ++q) {
-                if (jj[q] < nvec && vec_max(r[q], T()) >= bound) {
+        for (int e0 = warp * 8; e0 < nflag; e0 += TK_WARPS * 8) {
+            const int e = e0 + (lane >> 2);
+            if (e >= nflag) continue;
+            const int ent = sh.flist[e];
+            for (int j = (ent >> 9) * TM_U * TK_THREADS + (ent & 511) + (lane & 3) * TK_THREADS; j < nvec;
+                 j += SEG * TM_U * TK_THREADS) {
+                const uint4 r = __ldcg(rv + j);
+                if (vec_max(r, T()) >= bound) {
                     float x[N];
-                    unpack(r[q], x);
+                    unpack(r, x);
 #pragma unroll
-                    for (int e = 0; e < N; ++e)
-                        if (x[e] >= bound) append(x[e], jj[q] * N + e, cval, cidx, count, overflow);
+                    for (int q = 0; q < N; ++q)
+                        if (x[q] >= bound) append(x[q], j * N + q, cval, cidx, count, overflow);
                 }
             }
-        }
-        if (nvec > TK_THREADS * 32) {                  // rows longer than one vector per lane and share
-            for (int f = warp; f < nflag; f += TK_WARPS)
-                for (int j = (int)sh.flist[f] + TK_THREADS * (lane + 32); j < nvec; j += TK_THREADS * 32) {
-                    const uint4 r = __ldcg(rv + j);
-                    if (vec_max(r, T()) >= bound) {
-                        float x[N];
-                        unpack(r, x);
-#pragma unroll
-                        for (int e = 0; e < N; ++e)
-                            if (x[e] >= bound) append(x[e], j * N + e, cval, cidx, count, overflow);
-                    }
-                }
         }
     } else {
         for (int f = warp; f < nflag; f += TK_WARPS)
-            for (int v = (int)sh.flist[f] + TK_THREADS * lane; v < V; v += TK_THREADS * 32) {
+            for (int v = (int)(sh.flist[f] & 511) + TK_THREADS * lane; v < V; v += TK_THREADS * 32) {
                 const float x = to_float(row[v]);
                 if (x >= bound) append(x, v, cval, cidx, count, overflow);
             }
@@ -283,7 +280,8 @@ __global__ void __launch_bounds__(TK_THREADS, 2) verify_topk_kernel(const Verify
     const int rth = (k + TK_WARPS - 1) / TK_WARPS;
     for (int rr = 0; rr < nrows; ++rr) {
         // ---- pass 1: the row's maximum and a lower bound on its k-th largest
-        const float my_max = thread_max<T, VEC>(rows[rr], V, tid);
+        float seg[SEG];
+        const float my_max = thread_max<T, VEC>(rows[rr], V, tid, seg);
         const float wr = warp_rth_largest(my_max, rth, lane);
         float wm;
         asm("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(wm) : "f"(my_max));
@@ -295,14 +293,14 @@ __global__ void __launch_bounds__(TK_THREADS, 2) verify_topk_kernel(const Verify
         // ---- pass 2: candidates at or above the bound
         float* cv = cval + rr * CAP;
         int* ci = cidx + rr * CAP;
-        filter_row<T, VEC>(rows[rr], V, bound, my_max, cv, ci, &sh.count[rr], &sh.overflow[rr], sh, tid);
+        filter_row<T, VEC>(rows[rr], V, bound, seg, cv, ci, &sh.count[rr], &sh.overflow[rr], sh, tid);
         __syncthreads();
         if (sh.overflow[rr]) {                         // block-uniform: the bound was too loose
             const T* row = rows[rr];
             const float kth = radix_kth_largest([row](int v) { return to_float(row[v]); }, V, k, sh, tid);
             if (tid == 0) { sh.count[rr] = 0; sh.overflow[rr] = 0; }
             __syncthreads();
-            filter_row<T, VEC>(row, V, kth, my_max, cv, ci, &sh.count[rr], &sh.overflow[rr], sh, tid);
+            filter_row<T, VEC>(row, V, kth, seg, cv, ci, &sh.count[rr], &sh.overflow[rr], sh, tid);
             __syncthreads();
         }
 
