@@ -113,9 +113,21 @@ __device__ __forceinline__ void append(float x, int idx, float* cval, int* cidx,
     else *overflow = 1;
 }
 
+// Exclusive prefix of cnt over the warp, the warp's total in `total`.
+__device__ __forceinline__ int warp_excl_scan(int cnt, int lane, int& total) {
+    int incl = cnt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    total = __shfl_sync(0xffffffffu, incl, 31);
+    return incl - cnt;
+}
+
 // Pass 2: every logit at or above the bound goes into the candidate buffer.  Only the sub-shares
 // whose maximum reached the bound are read again (from L2): four lanes per flagged sub-share, one
-// vector each.
+// vector each.  List slots and buffer slots are claimed once per warp.
 template <typename T, bool VEC>
 __device__ __forceinline__ void filter_row(const T* __restrict__ row, int V, float bound, const float (&seg)[SEG],
                                            float* cval, int* cidx, int* count, int* overflow, TkShared& sh, int tid) {
@@ -123,29 +135,55 @@ __device__ __forceinline__ void filter_row(const T* __restrict__ row, int V, flo
     const int lane = tid & 31, warp = tid >> 5;
     if (tid == 0) sh.nflag = 0;
     __syncthreads();
+    {
+        unsigned mask = 0;
 #pragma unroll
-    for (int s = 0; s < (VEC ? SEG : 1); ++s)
-        if (seg[s] >= bound) sh.flist[atomicAdd(&sh.nflag, 1)] = (unsigned short)(tid | (s << 9));
+        for (int s = 0; s < (VEC ? SEG : 1); ++s) mask |= (seg[s] >= bound ? 1u : 0u) << s;
+        int total, base = 0;
+        int pos = warp_excl_scan(__popc(mask), lane, total);
+        if (total) {                                   // warp-uniform
+            if (lane == 31) base = atomicAdd(&sh.nflag, total);
+            pos += __shfl_sync(0xffffffffu, base, 31);
+            for (; mask; mask &= mask - 1) sh.flist[pos++] = (unsigned short)(tid | ((__ffs(mask) - 1) << 9));
+        }
+    }
     __syncthreads();
     const int nflag = sh.nflag;
     if constexpr (VEC) {
-        static_assert(TM_U == 4 && TK_THREADS == 512, "entry packing and lane mapping");
+        static_assert(32 % TM_U == 0 && TK_THREADS == 512 && SEG <= 8, "entry packing and lane mapping");
+        constexpr int EPT = 32 / TM_U;                 // entries a warp reads per trip
         const int nvec = V / N;
         const uint4* rv = reinterpret_cast<const uint4*>(row);
-        for (int e0 = warp * 8; e0 < nflag; e0 += TK_WARPS * 8) {
-            const int e = e0 + (lane >> 2);
-            if (e >= nflag) continue;
-            const int ent = sh.flist[e];
-            for (int j = (ent >> 9) * TM_U * TK_THREADS + (ent & 511) + (lane & 3) * TK_THREADS; j < nvec;
-                 j += SEG * TM_U * TK_THREADS) {
-                const uint4 r = __ldcg(rv + j);
-                if (vec_max(r, T()) >= bound) {
-                    float x[N];
+        for (int e0 = warp * EPT; e0 < nflag; e0 += TK_WARPS * EPT) {        // warp-uniform trip count
+            const int e = e0 + lane / TM_U;
+            int j = nvec;
+            if (e < nflag) {
+                const int ent = sh.flist[e];
+                j = (ent >> 9) * TM_U * TK_THREADS + (ent & 511) + (lane % TM_U) * TK_THREADS;
+            }
+            while (__any_sync(0xffffffffu, j < nvec)) {
+                float x[N];
+                unsigned hits = 0;
+                if (j < nvec) {
+                    const uint4 r = __ldcg(rv + j);
                     unpack(r, x);
 #pragma unroll
-                    for (int q = 0; q < N; ++q)
-                        if (x[q] >= bound) append(x[q], j * N + q, cval, cidx, count, overflow);
+                    for (int q = 0; q < N; ++q) hits |= (x[q] >= bound ? 1u : 0u) << q;
                 }
+                int total, base = 0;
+                int pos = warp_excl_scan(__popc(hits), lane, total);
+                if (total) {
+                    if (lane == 31) base = atomicAdd(count, total);
+                    pos += __shfl_sync(0xffffffffu, base, 31);
+#pragma unroll
+                    for (int q = 0; q < N; ++q)
+                        if (hits & (1u << q)) {
+                            if (pos < CAP) { cval[pos] = x[q]; cidx[pos] = j * N + q; }
+                            else *overflow = 1;
+                            ++pos;
+                        }
+                }
+                j += SEG * TM_U * TK_THREADS;
             }
         }
     } else {
