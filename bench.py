@@ -145,7 +145,7 @@ def algorithmic_bytes(cfg: wl.Workload, lens: np.ndarray) -> int:
 
 
 # ----------------------------------------------------------------------------------------- CPU arm
-def oracle_sample_rate(cfg: wl.Workload, inp: dict, budget_s: float, head=None):
+def oracle_sample_rate(cfg: wl.Workload, inp: dict, budget_s: float, head=None, top_k=None):
     """Times the CPU oracle (as it stands) on leading batch rows until `budget_s` is used.
     Returns (tokens/s, rows used, seconds, threads)."""
     from oracle import specdec_oracle as orc
@@ -159,7 +159,7 @@ def oracle_sample_rate(cfg: wl.Workload, inp: dict, budget_s: float, head=None):
             a = orc.accept_head(head["hidden"][sl], head["blocks"], head["w_out"], float(head["b_out"]))
             orc.stop_rule(a.astype(np.float32), cfg.h, lens[sl])
         orc.verify_correct(inp["target_logits"][sl], inp["draft_logits"][sl], inp["cand_tokens"][sl], lens[sl],
-                           inp["uniforms"][sl], inp["temperature"])
+                           inp["uniforms"][sl], inp["temperature"], top_k=top_k)
         tokens += int(lens[sl].sum())
         rows = sl.stop
     dt = time.perf_counter() - t0
@@ -250,8 +250,12 @@ def run_ours(args, cfg):
         specdec.specdec_stop(ctx, head_prob, cfg.h, d["cand_len"], stop_pos)
         if ev:
             ev[0].record()
-        specdec.specdec_verify_correct(ctx, d["target_logits"], d["draft_logits"], d["cand_tokens"], d["cand_len"],
-                                       d["uniforms"], T, n_out, t_out, flags=args.kernel)
+        if args.top_k > 0:
+            specdec.specdec_verify_correct_topk(ctx, d["target_logits"], d["draft_logits"], d["cand_tokens"],
+                                                d["cand_len"], d["uniforms"], T, args.top_k, n_out, t_out)
+        else:
+            specdec.specdec_verify_correct(ctx, d["target_logits"], d["draft_logits"], d["cand_tokens"], d["cand_len"],
+                                           d["uniforms"], T, n_out, t_out, flags=args.kernel)
         if ev:
             ev[1].record()
 
@@ -300,7 +304,7 @@ def run_ours(args, cfg):
         specdec.specdec_verify_correct_host(ctx, host["target_logits"], host["draft_logits"], host["cand_tokens"],
                                             host["cand_len"], host["uniforms"], T, h_n, h_t, flags=args.kernel)
 
-    if args.no_e2e:
+    if args.no_e2e or args.top_k > 0:               # the host-buffer entry point has no top-k form
         e2e_steps = 0
         e2e_ms = float("nan")
     else:
@@ -333,15 +337,19 @@ def run_ours(args, cfg):
         "roofline": {"kernel": "verify/correct", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
                      "frac_of_nominal_8TBs": achieved / 8000.0, "algorithmic_bytes": alg, "kernel_ms": verify_ms,
-                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name) if args.kernel == 0 else None},
+                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name) if args.kernel == 0 and args.top_k == 0 else None},
         "parts_ms": {"head": head_ms, "stop": stop_ms, "verify": verify_ms},
         "roofline_head": {"kernel": "acceptance head (2 x [M,4096]x[4096,4096] bf16 GEMM)", "bound": "tensor",
                           "achieved": head_flops / (head_ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"],
                           "unit": "TFLOP/s", "frac": head_flops / (head_ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                           "peak_source": peaks["source"] + " cuBLAS bf16 (sustained)"},
     }
+    if args.top_k > 0:
+        line["config"]["top_k"] = args.top_k
+        line["roofline"]["kernel"] = f"verify/correct, top-k {args.top_k}"
+        line["e2e"] = None
     if world == 1 and not args.no_cpu_baseline:
-        rate, rows, dt, cores = oracle_sample_rate(cfg, inp, args.cpu_budget, hd)
+        rate, rows, dt, cores = oracle_sample_rate(cfg, inp, args.cpu_budget, hd, args.top_k or None)
         line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"first {rows} of {cfg.B} batch rows of {cfg.name}, {dt:.1f} s"}
     print(json.dumps(line), flush=True)
@@ -358,6 +366,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(wl.CONFIGS))
     ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 direct, 2 stream")
+    ap.add_argument("--top-k", type=int, default=0,
+                    help="verify under top-k sampling (the paper's runs use 50); 0 = whole vocabulary, the headline workload")
     ap.add_argument("--cpu-budget", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
