@@ -54,10 +54,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait: on exhaustion a status bit is set and execution simply continues, so every
 // thread still reaches the barriers and the tensor-memory release below.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status) {
-    for (uint32_t it = 0; it < WAIT_POLLS; ++it)
+// `budget` is the calling thread's poll allowance: after one give-up the later waits of that thread
+// are short, so a broken pipeline drains in about a second instead of one limit per wait.
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status, uint32_t& budget) {
+    for (uint32_t it = 0; it < budget; ++it)
         if (mbar_try_wait(bar, parity)) return;
     atomicOr(status, SPECDEC_DATA_WAIT_LIMIT);
+    budget = 1024;
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
@@ -134,6 +137,7 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nkb = P.d / BK;
     const int ntn = P.d / BN, ntiles = ntn * ((P.M + BM - 1) / BM);
+    uint32_t budget = WAIT_POLLS;
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
@@ -164,7 +168,7 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
                 const int m0 = (t / ntn) * BM, n0 = (t % ntn) * BN;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    mbar_wait(empty0 + 8 * stage, phase ^ 1u, P.status);
+                    mbar_wait(empty0 + 8 * stage, phase ^ 1u, P.status, budget);
                     const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
                     mbar_expect_tx(full0 + 8 * stage, C::STAGE_BYTES);
                     tma_load_2d(a, &mapX, kb * BK, m0, full0 + 8 * stage);
@@ -180,11 +184,11 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             uint32_t stage = 0, phase = 0, it = 0;
             for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
                 const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
-                mbar_wait(tempty0 + 8 * buf, use ^ 1u, P.status);      // epilogue has drained this accumulator
+                mbar_wait(tempty0 + 8 * buf, use ^ 1u, P.status, budget);      // epilogue has drained this accumulator
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t acc = tmem + buf * BN;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    mbar_wait(full0 + 8 * stage, phase, P.status);
+                    mbar_wait(full0 + 8 * stage, phase, P.status, budget);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
 #pragma unroll
@@ -212,7 +216,7 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             uint4 xv[4], xn[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) xn[j] = row_ok ? __ldg(xrow + (half * CH) * 4 + j) : make_uint4(0, 0, 0, 0);
-            mbar_wait(tfull0 + 8 * buf, use, P.status);
+            mbar_wait(tfull0 + 8 * buf, use, P.status, budget);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             float dot = 0.f;
 #pragma unroll 1

@@ -51,6 +51,25 @@ def test_head_small_shapes(d, depth, with_bias, rows):
     ctx.close()
 
 
+@pytest.mark.parametrize("rows,d,depth", [((13, 47), 256, 1), ((13, 47), 512, 2), ((25, 31), 768, 2), ((64, 16), 1024, 3)],
+                         ids=["611x256", "611x512", "775x768", "1024x1024"])
+def test_head_many_row_tiles(rows, d, depth):
+    """Several row tiles with a ragged last one, widths up to 1024 and depth up to 3: every CTA gets
+    more than one tile at the larger sizes, which exercises the double-buffered accumulator and the
+    stage ring across tiles; the call is repeatable bit for bit."""
+    B, K = rows
+    ctx = specdec.Context(B, K, max_d=d)
+    hidden, Ws, bs, w_out, b_out = _head_problem(300 + d + depth, B, K, d, depth, True, std=0.02)
+    got = _run_head(ctx, hidden, Ws, bs, w_out, b_out)
+    want = orc.accept_head(hidden, list(zip(Ws, bs)), w_out, b_out)
+    err = np.abs(got - want) / want
+    assert err.max() <= HEAD_RTOL, (err.max(), np.argmax(err), got.ravel()[:4], want.ravel()[:4])
+    assert want.std() > 1e-3
+    got2 = _run_head(ctx, hidden, Ws, bs, w_out, b_out)
+    assert np.array_equal(got, got2)
+    ctx.close()
+
+
 def test_head_reduces_to_logistic_regression_when_weights_are_zero():
     B, K, d = 4, 40, 256
     ctx = specdec.Context(B, K, max_d=d)
