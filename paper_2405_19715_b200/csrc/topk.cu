@@ -168,7 +168,7 @@ __device__ __forceinline__ void filter_row(const T* __restrict__ row, int V, flo
                     const uint4 r = __ldcg(rv + j);
                     unpack(r, x);
 #pragma unroll
-                    for (int q = 0; q < N; ++q) hits |= (x[q] >= bound ? 1u : 0u) << q;
+                    for (int q = 0; q < N; ++q) hits |= (x[q] >= bound && x[q] > -INFINITY ? 1u : 0u) << q;   // masked (-inf) logits are never candidates
                 }
                 int total, base = 0;
                 int pos = warp_excl_scan(__popc(hits), lane, total);
@@ -190,7 +190,7 @@ __device__ __forceinline__ void filter_row(const T* __restrict__ row, int V, flo
         for (int f = warp; f < nflag; f += TK_WARPS)
             for (int v = (int)(sh.flist[f] & 511) + TK_THREADS * lane; v < V; v += TK_THREADS * 32) {
                 const float x = to_float(row[v]);
-                if (x >= bound) append(x, v, cval, cidx, count, overflow);
+                if (x >= bound && x > -INFINITY) append(x, v, cval, cidx, count, overflow);
             }
     }
 }

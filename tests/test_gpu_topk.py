@@ -91,3 +91,27 @@ def test_topk_adversarial_order_uses_the_exact_select():
     out = _run(ctx, flat, 50)
     assert ctx.device_status() == specdec.DATA_TOPK_TIES and np.all(out["n_accepted"] == -1)
     ctx.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_topk_with_a_masked_vocabulary(dtype):
+    """Constrained decoding masks most logits with -inf: with fewer finite logits than k the filter keeps
+    exactly the finite ones (the -inf entries carry no probability), and nothing is flagged."""
+    B, K, V, k = 5, 3, 20000, 50
+    ctx = specdec.Context(B, K)
+    cfg = wl.Workload("mk", B=B, K=K, V=V, dtype=dtype, sigma_d=2.0, sigma_n=1.0, T=1.0, ragged=False, seed=321)
+    inp = wl.make_verify_inputs(cfg, threads=1)
+    rng = np.random.default_rng(9)
+    allowed = np.sort(rng.choice(V, size=10, replace=False))
+    neg = np.float32(-np.inf) if dtype == "f32" else np.uint16(0xFF80)
+    for name in ("target_logits", "draft_logits"):
+        a = inp[name]
+        keep = a[..., allowed].copy()
+        a[...] = neg
+        a[..., allowed] = keep
+    inp["cand_tokens"] = allowed[rng.integers(0, 10, size=(B, K))].astype(np.int32)
+    gpu = _run(ctx, inp, k)
+    rep = parity.classify_rows(inp, gpu, dtype="f32", check_probs=False, top_k=k)
+    assert rep["exact"] + rep["boundary_n"] + rep["boundary_token"] == B and ctx.device_status() == 0
+    assert np.all(np.isin(gpu["next_token"], allowed))
+    ctx.close()
