@@ -60,6 +60,9 @@ typedef enum {
                                     statistics and accept tests, a second for the draws           */
 #define SPECDEC_VERIFY_FUSED   3u /* the same pipeline in one launch: CTAs that run out of units
                                     stream the draws of rows that are already resolved             */
+#define SPECDEC_VERIFY_CLUSTER 4u /* small batches: a cluster of 2-8 CTAs per (row, position), each taking
+                                    a slice of the vocabulary, combined through distributed shared
+                                    memory; picked automatically while the units fit the SMs twice   */
 
 /*
  * Create a context on `device` able to serve calls with B <= max_B and K <= max_K.

@@ -40,7 +40,7 @@ int check_verify_args(specdec_ctx* ctx, const void* target, const void* draft, i
     if (dtype != SPECDEC_F32 && dtype != SPECDEC_BF16) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown dtype %d", dtype);
     if (B < 1 || K < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "verify_correct: B, K, V must be >= 1 (got %d, %d, %d)", B, K, V);
     if (!(T > 0.f) || !std::isfinite(T)) return fail(ctx, SPECDEC_EINVAL, "verify_correct: temperature must be positive and finite");
-    if (flags > SPECDEC_VERIFY_FUSED) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown flags %u", flags);
+    if (flags > SPECDEC_VERIFY_CLUSTER) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown flags %u", flags);
     if (B > ctx->max_B || K > ctx->max_K)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: B=%d K=%d exceed the context (max_B=%d max_K=%d)", B, K, ctx->max_B, ctx->max_K);
     if (V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: V=%d above 2^22", V);
@@ -181,12 +181,16 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
         // round trips; below that the one-CTA-per-unit kernel has the shorter critical path.
         const double bytes = 2.0 * B * (K + 1.0) * V * (dtype == SPECDEC_BF16 ? 2 : 4);
         kind = (stream_ok && bytes >= 512e6) ? SPECDEC_VERIFY_FUSED : SPECDEC_VERIFY_DIRECT;
+        // a handful of units: several CTAs per unit, each on a slice of the vocabulary
+        if (kind == SPECDEC_VERIFY_DIRECT && verify_cluster_size(p, dtype, ctx->sm_count) > 1) kind = SPECDEC_VERIFY_CLUSTER;
     }
     if (kind == SPECDEC_VERIFY_FUSED && K > 63) kind = SPECDEC_VERIFY_STREAM;     // row records hold n in 6 bits
-    if (kind != SPECDEC_VERIFY_DIRECT && !stream_ok)
+    if (kind != SPECDEC_VERIFY_DIRECT && kind != SPECDEC_VERIFY_CLUSTER && !stream_ok)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: streaming kernels need 16-byte aligned rows (V=%d)", V);
     int n_launch = 0;
-    cudaError_t e = kind == SPECDEC_VERIFY_FUSED    ? launch_verify_fused(p, dtype, ctx->sm_count, s, &n_launch)
+    const int csize = kind == SPECDEC_VERIFY_CLUSTER ? verify_cluster_size(p, dtype, ctx->sm_count) : 1;
+    cudaError_t e = kind == SPECDEC_VERIFY_CLUSTER  ? launch_verify_cluster(p, dtype, csize > 1 ? csize : 2, s, &n_launch)
+                    : kind == SPECDEC_VERIFY_FUSED  ? launch_verify_fused(p, dtype, ctx->sm_count, s, &n_launch)
                     : kind == SPECDEC_VERIFY_STREAM ? launch_verify_stream(p, dtype, ctx->sm_count, s, &n_launch)
                                                     : launch_verify_direct(p, dtype, s, &n_launch);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "verify_correct launch");

@@ -79,3 +79,6 @@ cudaError_t launch_shard_draw(const specdec_shard& sh, const float* stats_all, c
                               int rank, const int32_t* n_acc, const int32_t* lens, const float* uniforms,
                               const float* row_norm, float c, int B, int K, int32_t* next, float* rmass,
                               cudaStream_t s);
+// Cluster size the small-batch kernel would use for this problem (1: not worth it).
+int verify_cluster_size(const VerifyParams& p, specdec_dtype dtype, int sm_count);
+cudaError_t launch_verify_cluster(const VerifyParams& p, specdec_dtype dtype, int C, cudaStream_t s, int* n_launch);

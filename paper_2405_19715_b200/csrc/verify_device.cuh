@@ -506,21 +506,19 @@ __device__ __forceinline__ int draw_select(const VerifyParams& P, const T* __res
     return tok;
 }
 
-// Block-wide inverse-CDF draw over the rows of one unit, read from global memory (L2).
-// A slab is the 32*EPV consecutive elements one warp covers with one vector per lane; slab
-// sums are fp32, everything above them is fp64.  Leaves the token in sh.token and the total
-// mass in sh.total.  All `nthreads` threads (tid 0..nthreads-1, whole warps) must call; uses
-// named barrier `bar_id`.
+// First half of a block-wide draw: the fp32 sum of the weights of every slab of the rows (read from
+// global memory, L2) into slab_sum.  A slab is the 32*EPV consecutive elements one warp covers
+// with one vector per lane.  All `nthreads` threads (tid 0..nthreads-1, whole warps) must call; the
+// caller synchronises before slab_sum is read.
 template <typename T, bool VEC>
-__device__ void unit_draw(const VerifyParams& P, const T* __restrict__ trow, const T* __restrict__ drow, int mode,
-                          float u01, UnitShared& sh, float* __restrict__ slab_sum, int tid, int nthreads, int bar_id,
-                          double tau_abs = -1.0) {
+__device__ __forceinline__ void unit_slabs(const VerifyParams& P, const T* __restrict__ trow,
+                                           const T* __restrict__ drow, int mode, const Norm np, const Norm nq,
+                                           float* __restrict__ slab_sum, int tid, int nthreads) {
     constexpr int N = Elem<T>::EPV;
     const int V = P.V;
     const int nvec = (V + N - 1) / N;
     const int nslab = (nvec + 31) / 32;
     const int warp = tid >> 5, lane = tid & 31, nwarp = nthreads >> 5;
-    const Norm np = sh.np, nq = sh.nq;
     float xt[N], xd[N], w[N];
 #pragma unroll
     for (int k = 0; k < N; ++k) xd[k] = 0.f;
@@ -570,6 +568,34 @@ __device__ void unit_draw(const VerifyParams& P, const T* __restrict__ trow, con
             if (lane == 0) slab_sum[s] = ls;
         }
     }
+}
+
+// Total of the slab sums in fp64, by one full warp, added in the order draw_select adds them (so the
+// two agree bit for bit).
+__device__ __forceinline__ double slab_total(const float* __restrict__ slab_sum, int nslab, int lane) {
+    const int per = (nslab + 31) / 32;
+    const int s0 = min(lane * per, nslab), s1 = min(s0 + per, nslab);
+    double mine = 0.0;
+    for (int s = s0; s < s1; ++s) mine += (double)slab_sum[s];
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    return __shfl_sync(0xffffffffu, incl, 31);
+}
+
+// Block-wide inverse-CDF draw over the rows of one unit: slab sums in fp32, everything above them
+// in fp64.  Leaves the token in sh.token and the total mass in sh.total.  All `nthreads` threads
+// (tid 0..nthreads-1, whole warps) must call; uses named barrier `bar_id`.
+template <typename T, bool VEC>
+__device__ void unit_draw(const VerifyParams& P, const T* __restrict__ trow, const T* __restrict__ drow, int mode,
+                          float u01, UnitShared& sh, float* __restrict__ slab_sum, int tid, int nthreads, int bar_id,
+                          double tau_abs = -1.0) {
+    const int warp = tid >> 5, lane = tid & 31;
+    const Norm np = sh.np, nq = sh.nq;
+    unit_slabs<T, VEC>(P, trow, drow, mode, np, nq, slab_sum, tid, nthreads);
     bar_sync(bar_id, nthreads);
 
     if (warp == 0) {

@@ -8,8 +8,8 @@ pytestmark = pytest.mark.gpu
 from paper_2405_19715_b200 import specdec, workloads as wl  # noqa: E402
 from tests import parity  # noqa: E402
 
-KERNELS = [specdec.VERIFY_DIRECT, specdec.VERIFY_STREAM, specdec.VERIFY_FUSED]
-KERNEL_IDS = ["direct", "stream", "fused"]
+KERNELS = [specdec.VERIFY_DIRECT, specdec.VERIFY_STREAM, specdec.VERIFY_FUSED, specdec.VERIFY_CLUSTER]
+KERNEL_IDS = ["direct", "stream", "fused", "cluster"]
 
 
 @pytest.fixture(scope="module")
@@ -47,7 +47,7 @@ def _random_problem(seed, B, K, V, dtype, T=1.0, sigma_n=1.0, ragged=True):
 @pytest.mark.parametrize("K", [1, 2, 16])
 def test_small_shapes(ctx, V, K, dtype, flags):
     inp = _random_problem(1000 + V + K, B=5, K=K, V=V, dtype=dtype, T=0.9)
-    if flags != specdec.VERIFY_DIRECT and not _stream_ok(inp):
+    if flags in (specdec.VERIFY_STREAM, specdec.VERIFY_FUSED) and not _stream_ok(inp):
         pytest.skip("rows not 16-byte aligned: served by the direct kernel")
     gpu = parity.run_gpu_verify(ctx, inp, flags)
     rep = parity.classify_rows(inp, gpu, dtype="f32")      # bf16 inputs are widened exactly: same bar
