@@ -38,7 +38,7 @@ def _topk_tokens(inp, cfg, k):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-@pytest.mark.parametrize("V,k", [(7, 3), (33, 50), (1000, 50), (3000, 50), (4104, 1), (20000, 50), (32000, 256)])
+@pytest.mark.parametrize("V,k", [(7, 3), (33, 50), (1000, 50), (3000, 50), (4104, 1), (20000, 50), (32000, 256), (200000, 50), (262144, 7)])
 def test_topk_small_shapes(V, k, dtype):
     B, K = 6, 5
     ctx = specdec.Context(B, K)
