@@ -18,6 +18,9 @@
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the
  *     legacy default stream) unless stated otherwise; outputs are valid once the
  *     stream has been synchronised.
+ *   - Every call that takes a context makes that context's GPU the calling thread's current
+ *     device (cudaSetDevice) and leaves it so; a process that drives several GPUs creates one
+ *     context per GPU.
  *   - A context owns small scratch buffers.  Two calls that use the same context must
  *     not overlap on the GPU (use one context per stream).
  *   - Return value: SPECDEC_OK or an error code; specdec_last_error() gives a message.

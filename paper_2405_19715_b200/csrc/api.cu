@@ -31,6 +31,12 @@ int cuda_fail(specdec_ctx* ctx, cudaError_t e, const char* what) {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Every entry point runs on the context's GPU, whichever device the calling thread had current.
+int use_device(specdec_ctx* ctx) {
+    cudaError_t e = cudaSetDevice(ctx->device);
+    return e == cudaSuccess ? SPECDEC_OK : cuda_fail(ctx, e, "cudaSetDevice");
+}
+
 int check_verify_args(specdec_ctx* ctx, const void* target, const void* draft, int dtype, const int32_t* tokens,
                       const float* uniforms, float T, int B, int K, int V, const int32_t* n_acc,
                       const int32_t* next, uint32_t flags) {
@@ -44,7 +50,7 @@ int check_verify_args(specdec_ctx* ctx, const void* target, const void* draft, i
     if (B > ctx->max_B || K > ctx->max_K)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: B=%d K=%d exceed the context (max_B=%d max_K=%d)", B, K, ctx->max_B, ctx->max_K);
     if (V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: V=%d above 2^22", V);
-    return SPECDEC_OK;
+    return use_device(ctx);
 }
 
 }  // namespace
@@ -120,6 +126,7 @@ uint64_t specdec_launch_count(const specdec_ctx* ctx) { return ctx ? ctx->launch
 
 int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits) {
     if (!ctx) return SPECDEC_EINVAL;
+    if (int rc = use_device(ctx)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint32_t host = 0;
     CU(ctx, cudaMemcpyAsync(&host, ctx->status, sizeof(host), cudaMemcpyDeviceToHost, s));
@@ -453,6 +460,7 @@ int specdec_stop(specdec_ctx* ctx, const float* accept_prob, const int32_t* cand
     if (!accept_prob || !stop_pos) return fail(ctx, SPECDEC_EINVAL, "stop: null pointer argument");
     if (B < 1 || K < 1) return fail(ctx, SPECDEC_EINVAL, "stop: B and K must be >= 1");
     if (h != h) return fail(ctx, SPECDEC_EINVAL, "stop: threshold is NaN");
+    if (int rc = use_device(ctx)) return rc;
     cudaError_t e = launch_stop(accept_prob, cand_len, h, B, K, stop_pos, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "stop launch");
     ctx->launches += 1;
@@ -465,6 +473,7 @@ int specdec_stop_step(specdec_ctx* ctx, const float* accept_prob_step, float* p_
     if (!accept_prob_step || !p_hat || !stop) return fail(ctx, SPECDEC_EINVAL, "stop_step: null pointer argument");
     if (B < 1) return fail(ctx, SPECDEC_EINVAL, "stop_step: B must be >= 1");
     if (h != h) return fail(ctx, SPECDEC_EINVAL, "stop_step: threshold is NaN");
+    if (int rc = use_device(ctx)) return rc;
     cudaError_t e = launch_stop_step(accept_prob_step, p_hat, h, B, stop, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "stop_step launch");
     ctx->launches += 1;
@@ -473,6 +482,7 @@ int specdec_stop_step(specdec_ctx* ctx, const float* accept_prob_step, float* p_
 
 int specdec_selftest_wait_limit(specdec_ctx* ctx, void* stream) {
     if (!ctx) return SPECDEC_EINVAL;
+    if (int rc = use_device(ctx)) return rc;
     cudaError_t e = launch_wait_limit_selftest(ctx->status, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "selftest launch");
     ctx->launches += 1;
