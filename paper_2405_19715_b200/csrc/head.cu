@@ -109,6 +109,7 @@ __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w &
 
 struct BlockParams {
     const __nv_bfloat16* X;      // [M, d] input of the block (also the residual)
+    const __nv_bfloat16* W;      // [d, d] weights, (out, in)
     const __nv_bfloat16* bias;   // [d] or null
     __nv_bfloat16* Y;            // [M, d] output, null for the last block
     const __nv_bfloat16* w_out;  // [d], last block only
@@ -116,6 +117,10 @@ struct BlockParams {
     int M, d;
     int sm_count;
     uint32_t* status;
+    // few-row path, last block: the CTA that finishes last adds the partial dots and applies the sigmoid
+    int32_t* done_ctr;
+    float* accept_prob;
+    float b_out;
 };
 
 // Persistent: CTA c works on tiles c, c + grid, ... (column tile fastest).  The accumulator is
@@ -266,6 +271,165 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The block for a few rows (Algorithm 1 runs the head once per drafted token: M = number of
+// sequences).  With M <= 8 the block is a stream of the 2 d^2 weight bytes against rows that fit in
+// shared memory, so it runs on the CUDA cores at HBM rate: a CTA owns 32 output columns, each of
+// its 8 warps 4 of them; lanes walk along k (coalesced 512-byte pieces of a weight row, 16 of them
+// in flight per lane), every row of X is read from shared memory once per four columns, and the
+// per-lane partial sums are reduced with shuffles.  The epilogue is the one of the tensor path.
+// packed fp32 pairs: one instruction, two multiply-adds (the two halves are two output columns)
+using f2 = unsigned long long;
+__device__ __forceinline__ f2 pack2(float a, float b) {
+    f2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f2 v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c) {
+    f2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+constexpr int GV_WARPS = 8, GV_COLS = 4, GV_UNROLL = 4;
+constexpr int GV_THREADS = GV_WARPS * 32, GV_TILE = GV_WARPS * GV_COLS;
+
+template <int MR>                  // rows held (a power of two >= M); missing rows are zero
+__global__ void __launch_bounds__(GV_THREADS) head_rows_kernel(const BlockParams P) {
+    extern __shared__ uint4 xs[];                      // [MR][d / 8]: the rows of X, bf16
+    __shared__ float dots[GV_WARPS][MR];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int d = P.d, dv = d >> 3, nchunk = d >> 8;   // a chunk: 256 k-elements, one 16-byte vector per lane
+    const int n0 = blockIdx.x * GV_TILE + warp * GV_COLS;
+    const uint4* wrow[GV_COLS];
+#pragma unroll
+    for (int c = 0; c < GV_COLS; ++c) wrow[c] = reinterpret_cast<const uint4*>(P.W + (size_t)(n0 + c) * d) + lane;
+
+    // first round of weight loads, then the rows of X while those are in flight
+    uint4 wv[GV_UNROLL][GV_COLS];
+#pragma unroll
+    for (int u = 0; u < GV_UNROLL; ++u)
+#pragma unroll
+        for (int c = 0; c < GV_COLS; ++c) wv[u][c] = u < nchunk ? __ldcs(wrow[c] + u * 32) : make_uint4(0, 0, 0, 0);
+    for (int i = tid; i < MR * dv; i += GV_THREADS) {
+        const int m = i / dv;
+        xs[i] = m < P.M ? __ldg(reinterpret_cast<const uint4*>(P.X) + (size_t)m * dv + (i - m * dv)) : make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+
+    f2 acc2[GV_COLS / 2][MR];                          // columns (2p, 2p + 1) side by side
+#pragma unroll
+    for (int p = 0; p < GV_COLS / 2; ++p)
+#pragma unroll
+        for (int m = 0; m < MR; ++m) acc2[p][m] = pack2(0.f, 0.f);
+    for (int ch0 = 0; ch0 < nchunk; ch0 += GV_UNROLL) {
+        uint4 cur[GV_UNROLL][GV_COLS];
+#pragma unroll
+        for (int u = 0; u < GV_UNROLL; ++u)
+#pragma unroll
+            for (int c = 0; c < GV_COLS; ++c) {
+                cur[u][c] = wv[u][c];
+                const int nx = ch0 + GV_UNROLL + u;    // the next round, issued before this one is consumed
+                wv[u][c] = nx < nchunk ? __ldcs(wrow[c] + nx * 32) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+        for (int u = 0; u < GV_UNROLL; ++u) {
+            if (ch0 + u >= nchunk) break;
+            f2 wp[GV_COLS / 2][8];
+#pragma unroll
+            for (int p = 0; p < GV_COLS / 2; ++p) {
+                const uint32_t* wa = reinterpret_cast<const uint32_t*>(&cur[u][2 * p]);
+                const uint32_t* wb = reinterpret_cast<const uint32_t*>(&cur[u][2 * p + 1]);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    wp[p][2 * j] = pack2(bf16lo(wa[j]), bf16lo(wb[j]));
+                    wp[p][2 * j + 1] = pack2(bf16hi(wa[j]), bf16hi(wb[j]));
+                }
+            }
+#pragma unroll
+            for (int m = 0; m < MR; ++m) {
+                const uint4 xv = xs[m * dv + (ch0 + u) * 32 + lane];
+                const uint32_t* x32 = reinterpret_cast<const uint32_t*>(&xv);
+                float xf[8];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { xf[2 * j] = bf16lo(x32[j]); xf[2 * j + 1] = bf16hi(x32[j]); }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const f2 xx = pack2(xf[j], xf[j]);
+#pragma unroll
+                    for (int p = 0; p < GV_COLS / 2; ++p) acc2[p][m] = fma2(wp[p][j], xx, acc2[p][m]);
+                }
+            }
+        }
+    }
+    // sums over the lanes (every lane ends with all of them), then lane c * MR + m finishes element (m, n0 + c)
+    float mine = 0.f;
+#pragma unroll
+    for (int c = 0; c < GV_COLS; ++c)
+#pragma unroll
+        for (int m = 0; m < MR; ++m) {
+            float lo, hi;
+            unpack2(acc2[c >> 1][m], lo, hi);
+            float v = (c & 1) ? hi : lo;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+            if (lane == c * MR + m) mine = v;
+        }
+    float contrib = 0.f;
+    if (lane < GV_COLS * MR) {
+        const int c = lane / MR, m = lane - c * MR, n = n0 + c;
+        if (m < P.M) {
+            const float z = mine + (P.bias ? __bfloat162float(P.bias[n]) : 0.f);
+            const float y = __bfloat162float(P.X[(size_t)m * d + n]) + silu(z);
+            if (P.Y) P.Y[(size_t)m * d + n] = __float2bfloat16_rn(y);
+            if (P.w_out) contrib = y * __bfloat162float(P.w_out[n]);
+        }
+    }
+    if (P.partial) {                                   // last block: one partial dot per (row, CTA), in a fixed order
+#pragma unroll
+        for (int o = MR; o < GV_COLS * MR; o <<= 1) contrib += __shfl_xor_sync(0xffffffffu, contrib, o);
+        if (lane < MR) dots[warp][lane] = contrib;
+        __syncthreads();
+        const int nt = d / GV_TILE;
+        if (tid < MR && tid < P.M) {
+            float sum = 0.f;
+#pragma unroll
+            for (int w = 0; w < GV_WARPS; ++w) sum += dots[w][tid];
+            P.partial[(size_t)tid * nt + blockIdx.x] = sum;
+        }
+        // the last CTA to get here finishes the head: accept_prob[m] = sigmoid(sum_t partial[m, t] + b_out),
+        // a warp per row, added in a fixed order
+        __shared__ int last;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) last = (atomicAdd(P.done_ctr, 1) == (int)gridDim.x - 1);
+        __syncthreads();
+        if (last) {
+            __threadfence();
+            if (warp < P.M) {
+                float v = 0.f;
+                for (int t = lane; t < nt; t += 32) v += __ldcg(P.partial + (size_t)warp * nt + t);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == 0) P.accept_prob[warp] = 1.f / (1.f + __expf(-(v + P.b_out)));
+            }
+            if (tid == 0) *P.done_ctr = 0;             // ready for the next call
+        }
+    }
+}
+
+template <int MR>
+cudaError_t launch_rows(const BlockParams& p, cudaStream_t s) {
+    const size_t smem = (size_t)MR * p.d * 2;
+    if (smem > 40 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(head_rows_kernel<MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+    }
+    head_rows_kernel<MR><<<p.d / GV_TILE, GV_THREADS, smem, s>>>(p);
+    return cudaGetLastError();
+}
+
 // accept_prob[m] = sigmoid(sum_t partial[m, t] + b_out)
 __global__ void head_finish_kernel(const float* __restrict__ partial, int M, int nt, float b_out,
                                    float* __restrict__ accept_prob) {
@@ -369,6 +533,8 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
     // few rows (the online, one-token-per-call use): narrow column tiles so that the weight stream is
     // spread over many SMs; otherwise the widest tile the width allows
     const int BN = M <= 256 ? 64 : (d % 256 == 0 ? 256 : 128);
+    // a handful of rows: the weight stream on the CUDA cores (no tensor maps needed)
+    const bool rows_path = M <= 8 && d % 256 == 0 && d <= 8192;
     for (int k = 0; k < D; ++k) {
         const void* W = head->W[k];
         const void* bias = head->b ? head->b[k] : nullptr;
@@ -376,10 +542,11 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
             return fail(ctx, SPECDEC_EINVAL, "accept_head: weights and biases must be non-null and 16-byte aligned");
         const bool last = (k == D - 1);
         CUtensorMap mx, mw;
-        if (!make_map(&mx, x, (int)M, d, BM) || !make_map(&mw, W, d, d, BN))
+        if (!rows_path && (!make_map(&mx, x, (int)M, d, BM) || !make_map(&mw, W, d, d, BN)))
             return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
         BlockParams p;
         p.X = x;
+        p.W = static_cast<const __nv_bfloat16*>(W);
         p.bias = static_cast<const __nv_bfloat16*>(bias);
         p.Y = last ? nullptr : static_cast<__nv_bfloat16*>(ctx->act[k & 1]);
         p.w_out = last ? static_cast<const __nv_bfloat16*>(head->w_out) : nullptr;
@@ -388,14 +555,21 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
         p.d = d;
         p.sm_count = ctx->sm_count;
         p.status = ctx->status;
-        cudaError_t e = BN == 256 ? launch_block<256>(mx, mw, p, s)
+        p.done_ctr = ctx->task_ctl + 5;
+        p.accept_prob = accept_prob;
+        p.b_out = head->b_out;
+        cudaError_t e = rows_path ? (M <= 1 ? launch_rows<1>(p, s) : M <= 2 ? launch_rows<2>(p, s)
+                                     : M <= 4 ? launch_rows<4>(p, s) : launch_rows<8>(p, s))
+                        : BN == 256 ? launch_block<256>(mx, mw, p, s)
                         : BN == 128 ? launch_block<128>(mx, mw, p, s) : launch_block<64>(mx, mw, p, s);
         if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
         ctx->launches += 1;
         x = p.Y;
     }
-    head_finish_kernel<<<(int)((M + 127) / 128), 128, 0, s>>>(ctx->head_partial, (int)M, 2 * d / BN, head->b_out, accept_prob);
-    ctx->launches += 1;
+    if (!rows_path) {
+        head_finish_kernel<<<(int)((M + 127) / 128), 128, 0, s>>>(ctx->head_partial, (int)M, 2 * d / BN, head->b_out, accept_prob);
+        ctx->launches += 1;
+    }
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? SPECDEC_OK : fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
 }

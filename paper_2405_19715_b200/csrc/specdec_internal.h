@@ -18,7 +18,7 @@ struct specdec_ctx {
     uint32_t* status = nullptr;   // sticky SPECDEC_DATA_* bits
     float4* norms = nullptr;      // [max_B * (max_K+1)]  log2 normalisers {hi_p, lo_p, hi_q, lo_q} per position
     int2* tasks = nullptr;        // [max_B]              rows whose y' is still to be drawn: {b, n}
-    int32_t* task_ctl = nullptr;  // [8]                  two-launch path: {tasks, finished CTAs}; fused path: {-, -, -, head, finished}
+    int32_t* task_ctl = nullptr;  // [8]                  two-launch path: {tasks, finished CTAs}; fused path: {-, -, -, head, finished}; [5]: CTAs done in the few-row head block
     int32_t* task_ready = nullptr;// [max_B]              fused path: record {epoch:24, mode:2, n:6} of each resolved row
     uint32_t epoch = 0;
     uint64_t launches = 0;

@@ -70,6 +70,21 @@ def test_head_many_row_tiles(rows, d, depth):
     ctx.close()
 
 
+@pytest.mark.parametrize("rows", [1, 2, 3, 4, 5, 8])
+@pytest.mark.parametrize("d,depth,with_bias", [(256, 1, True), (512, 3, False), (4096, 2, True)])
+def test_head_few_rows(rows, d, depth, with_bias):
+    """At most 8 rows (one drafted token for a few sequences) take the weight-streaming kernel; row counts
+    that are not powers of two leave zero-padded rows."""
+    ctx = specdec.Context(rows, 1, max_d=d)
+    hidden, Ws, bs, w_out, b_out = _head_problem(700 + rows + d, rows, 1, d, depth, with_bias, std=0.02 if d > 512 else 0.05)
+    got = _run_head(ctx, hidden, Ws, bs, w_out, b_out)
+    want = orc.accept_head(hidden, list(zip(Ws, bs)), w_out, b_out)
+    err = np.abs(got - want) / want
+    assert err.max() <= HEAD_RTOL, (err.max(), got.ravel()[:4], want.ravel()[:4])
+    assert np.array_equal(got, _run_head(ctx, hidden, Ws, bs, w_out, b_out))
+    ctx.close()
+
+
 def test_head_reduces_to_logistic_regression_when_weights_are_zero():
     B, K, d = 4, 40, 256
     ctx = specdec.Context(B, K, max_d=d)
