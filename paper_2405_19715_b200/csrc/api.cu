@@ -33,6 +33,8 @@ size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Every entry point runs on the context's GPU, whichever device the calling thread had current.
 int use_device(specdec_ctx* ctx) {
+    int cur = -1;
+    if (cudaGetDevice(&cur) == cudaSuccess && cur == ctx->device) return SPECDEC_OK;   // the usual case, no driver call
     cudaError_t e = cudaSetDevice(ctx->device);
     return e == cudaSuccess ? SPECDEC_OK : cuda_fail(ctx, e, "cudaSetDevice");
 }
@@ -262,8 +264,7 @@ int specdec_sample(specdec_ctx* ctx, const void* logits, specdec_dtype dtype, co
     if (B < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "sample: B and V must be >= 1 (got %d, %d)", B, V);
     if (B > ctx->max_B) return fail(ctx, SPECDEC_EUNSUPPORTED, "sample: B=%d exceeds the context (max_B=%d)", B, ctx->max_B);
     if (top_k > 256 && top_k < V) return fail(ctx, SPECDEC_EINVAL, "sample: top_k must be <= 256, or <= 0 / >= V for none (got %d)", top_k);
-    cudaError_t e0 = cudaSetDevice(ctx->device);
-    if (e0 != cudaSuccess) return cuda_fail(ctx, e0, "cudaSetDevice");
+    if (int rc0 = use_device(ctx)) return rc0;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     ctx->epoch = (ctx->epoch + 1) & 0x3fffffffu;
     if ((ctx->epoch & 0xffffffu) == 0)
@@ -311,9 +312,7 @@ int check_shard_args(specdec_ctx* ctx, const specdec_shard* sh, float T, int B, 
         return fail(ctx, SPECDEC_EINVAL, "%s: columns [%d, %d + %d) do not lie in a vocabulary of %d", who, sh->v_offset, sh->v_offset, sh->V_shard, sh->V);
     if (!(T > 0.f) || !std::isfinite(T)) return fail(ctx, SPECDEC_EINVAL, "%s: temperature must be positive and finite", who);
     if (sh->V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "%s: V=%d above 2^22", who, sh->V);
-    cudaError_t e = cudaSetDevice(ctx->device);
-    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaSetDevice");
-    return SPECDEC_OK;
+    return use_device(ctx);
 }
 }  // namespace
 
