@@ -14,7 +14,7 @@ from oracle import specdec_oracle as orc
 from paper_2405_19715_b200 import specdec
 
 BOUNDARY = 1e-6
-PROB_RTOL = {"f32": 1e-5, "bf16": 2e-2}     # spec tolerances on probabilities
+PROB_RTOL = {"f32": 1e-5, "bf16": 2e-2}     # relative tolerances on probabilities by logit dtype
 
 
 to_torch = specdec.from_numpy

@@ -10,7 +10,7 @@ from oracle import specdec_oracle as orc  # noqa: E402
 from paper_2405_19715_b200 import specdec, workloads as wl  # noqa: E402
 from tests import parity  # noqa: E402
 
-HEAD_RTOL = 2e-2      # spec tolerance for bf16 head outputs
+HEAD_RTOL = 2e-2      # tolerance for head outputs computed from bf16 activations
 
 
 def _head_problem(seed, B, K, d, depth, with_bias, std=0.05):
