@@ -8,10 +8,12 @@ namespace {
 
 using namespace sd;
 
-constexpr int DIRECT_THREADS = 512;
 
-template <typename T, bool VEC>
-__global__ void __launch_bounds__(DIRECT_THREADS, 2) verify_direct_kernel(const VerifyParams P) {
+// DIRECT_THREADS threads per unit: 512 (two CTAs per SM) when the units fit the machine a few times
+// over, 256 (four per SM) for larger grids, where more resident units hide each unit's dependent
+// chain (accept test, draw, row counter) better than a shorter pass does.
+template <typename T, bool VEC, int DIRECT_THREADS>
+__global__ void __launch_bounds__(DIRECT_THREADS, 1024 / DIRECT_THREADS) verify_direct_kernel(const VerifyParams P) {
     constexpr int N = Elem<T>::EPV;
     extern __shared__ float slab_sum[];
     __shared__ UnitShared sh;
@@ -97,12 +99,19 @@ cudaError_t launch_t(const VerifyParams& p, cudaStream_t s) {
     const bool vec = (p.V % N == 0) && (reinterpret_cast<uintptr_t>(p.target) % 16 == 0) &&
                      (reinterpret_cast<uintptr_t>(p.draft) % 16 == 0);
     const int grid = p.B * (p.K + 1);
-    auto kern = vec ? verify_direct_kernel<T, true> : verify_direct_kernel<T, false>;
+    static const int sms = [] {
+        int dev = 0, n = 148;
+        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        return n;
+    }();
+    const bool small_ctas = grid >= 12 * sms;
+    auto kern = small_ctas ? (vec ? verify_direct_kernel<T, true, 256> : verify_direct_kernel<T, false, 256>)
+                           : (vec ? verify_direct_kernel<T, true, 512> : verify_direct_kernel<T, false, 512>);
     if (smem > 40 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
     }
-    kern<<<grid, DIRECT_THREADS, smem, s>>>(p);
+    kern<<<grid, small_ctas ? 256 : 512, smem, s>>>(p);
     return cudaGetLastError();
 }
 
