@@ -28,9 +28,9 @@ sys.path.insert(0, str(ROOT))
 
 from paper_2405_19715_b200 import workloads as wl  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one verify/correct launch (fused kernel), from the ncu capture
-# summarised in profiles/verify_fused_cfg4_B32_B128.md, scaled by units to the full workload.
-NCU_TRAFFIC_BYTES = {"cfg4": 2.3199e9}
+# dram__bytes_read.sum + dram__bytes_write.sum of one verify/correct launch (the kernel the library picks at this
+# size), from the ncu capture at half the batch summarised in profiles/verify_direct_cfg4_B128.md, scaled by units.
+NCU_TRAFFIC_BYTES = {"cfg4": 2.3044e9}
 
 METRIC = "verified candidate tokens/s"
 UNIT = "tokens/s"
@@ -365,7 +365,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(wl.CONFIGS))
-    ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 direct, 2 stream")
+    ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 one CTA per unit, 2 two-launch TMA pipeline, 3 fused TMA pipeline, 4 cluster per unit")
     ap.add_argument("--top-k", type=int, default=0,
                     help="verify under top-k sampling (the paper's runs use 50); 0 = whole vocabulary, the headline workload")
     ap.add_argument("--cpu-budget", type=float, default=12.0)

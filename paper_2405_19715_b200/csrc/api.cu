@@ -186,12 +186,10 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
     const bool stream_ok = verify_stream_supported(p, dtype);
     uint32_t kind = flags;
     if (kind == SPECDEC_VERIFY_AUTO) {
-        // The persistent pipeline pays off once the logits clearly exceed what the SMs can pull in a few
-        // round trips; below that the one-CTA-per-unit kernel has the shorter critical path.
-        const double bytes = 2.0 * B * (K + 1.0) * V * (dtype == SPECDEC_BF16 ? 2 : 4);
-        kind = (stream_ok && bytes >= 512e6) ? SPECDEC_VERIFY_FUSED : SPECDEC_VERIFY_DIRECT;
-        // a handful of units: several CTAs per unit, each on a slice of the vocabulary
-        if (kind == SPECDEC_VERIFY_DIRECT && verify_cluster_size(p, dtype, ctx->sm_count) > 1) kind = SPECDEC_VERIFY_CLUSTER;
+        // One CTA per unit (four 256-thread CTAs per SM on large grids) measured at or ahead of the
+        // persistent TMA pipelines at every size tried, so those stay selectable but are not picked here.
+        // A handful of units: several CTAs per unit, each on a slice of the vocabulary.
+        kind = verify_cluster_size(p, dtype, ctx->sm_count) > 1 ? SPECDEC_VERIFY_CLUSTER : SPECDEC_VERIFY_DIRECT;
     }
     if (kind == SPECDEC_VERIFY_FUSED && K > 63) kind = SPECDEC_VERIFY_STREAM;     // row records hold n in 6 bits
     if (kind != SPECDEC_VERIFY_DIRECT && kind != SPECDEC_VERIFY_CLUSTER && !stream_ok)
