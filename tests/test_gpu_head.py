@@ -70,7 +70,7 @@ def test_head_many_row_tiles(rows, d, depth):
     ctx.close()
 
 
-@pytest.mark.parametrize("rows", [1, 2, 3, 4, 5, 8, 9, 13, 16])
+@pytest.mark.parametrize("rows", [1, 2, 3, 4, 5, 8, 9, 13, 16, 17, 32, 33, 64, 65])
 @pytest.mark.parametrize("d,depth,with_bias", [(256, 1, True), (512, 3, False), (4096, 2, True)])
 def test_head_few_rows(rows, d, depth, with_bias):
     """At most 8 rows (one drafted token for a few sequences) take the weight-streaming kernel; row counts
