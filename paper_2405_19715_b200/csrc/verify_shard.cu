@@ -40,12 +40,13 @@ __device__ __forceinline__ const T* draft_row(const ShardRows& S, int K, int b, 
 // ---- phase 1 -----------------------------------------------------------------------------
 // record: {rs_p, s_p, rs_q, s_q, t_y, d_y, owned, 0}; t_y, d_y, owned are zero unless this rank
 // holds column y, so that summing the records of all ranks yields them exactly.
-template <typename T, bool VEC>
-__global__ void __launch_bounds__(SHARD_THREADS) shard_stats_kernel(ShardRows S, const int32_t* __restrict__ tokens,
+// THREADS: 512, or 256 (four CTAs per SM) on grids that cover the machine many times over.
+template <typename T, bool VEC, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS) shard_stats_kernel(ShardRows S, const int32_t* __restrict__ tokens,
                                                                     const int32_t* __restrict__ lens, float c, int B,
                                                                     int K, float* __restrict__ stats,
                                                                     uint32_t* __restrict__ status) {
-    __shared__ Acc wp[SHARD_THREADS / 32], wq[SHARD_THREADS / 32];
+    __shared__ Acc wp[THREADS / 32], wq[THREADS / 32];
     const int unit = blockIdx.x;
     const int i = unit / B, b = unit - i * B;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -73,13 +74,13 @@ __global__ void __launch_bounds__(SHARD_THREADS) shard_stats_kernel(ShardRows S,
         }
     }
     Acc ap = acc_init(), aq = acc_init();
-    unit_stats<T, VEC, SHARD_THREADS>(trow, drow, S.Vs, c, bonus, tid, ap, aq);
+    unit_stats<T, VEC, THREADS>(trow, drow, S.Vs, c, bonus, tid, ap, aq);
     ap = warp_merge(ap);
     aq = warp_merge(aq);
     if (lane == 0) { wp[warp] = ap; wq[warp] = aq; }
     __syncthreads();
     if (warp == 0) {
-        constexpr int NW = SHARD_THREADS / 32;
+        constexpr int NW = THREADS / 32;
         Acc a = lane < NW ? wp[lane] : acc_init(), q = lane < NW ? wq[lane] : acc_init();
         a = warp_merge(a);
         q = warp_merge(q);
@@ -275,17 +276,25 @@ ShardRows rows_of(const specdec_shard& sh) {
 
 }  // namespace
 
+template <typename T>
+void launch_stats_t(const specdec_shard& sh, const ShardRows& S, const int32_t* tokens, const int32_t* lens, float c,
+                    int B, int K, float* stats, uint32_t* status, cudaStream_t s) {
+    const int grid = B * (K + 1);
+    const bool vec = shard_vec<T>(sh), small = grid >= 12 * 148;
+    if (small) {
+        if (vec) shard_stats_kernel<T, true, 256><<<grid, 256, 0, s>>>(S, tokens, lens, c, B, K, stats, status);
+        else shard_stats_kernel<T, false, 256><<<grid, 256, 0, s>>>(S, tokens, lens, c, B, K, stats, status);
+    } else {
+        if (vec) shard_stats_kernel<T, true, 512><<<grid, 512, 0, s>>>(S, tokens, lens, c, B, K, stats, status);
+        else shard_stats_kernel<T, false, 512><<<grid, 512, 0, s>>>(S, tokens, lens, c, B, K, stats, status);
+    }
+}
+
 cudaError_t launch_shard_stats(const specdec_shard& sh, const int32_t* tokens, const int32_t* lens, float c, int B,
                                int K, float* stats, uint32_t* status, cudaStream_t s) {
     const ShardRows S = rows_of(sh);
-    const int grid = B * (K + 1);
-    if (sh.dtype == SPECDEC_BF16) {
-        if (shard_vec<__nv_bfloat16>(sh)) shard_stats_kernel<__nv_bfloat16, true><<<grid, SHARD_THREADS, 0, s>>>(S, tokens, lens, c, B, K, stats, status);
-        else shard_stats_kernel<__nv_bfloat16, false><<<grid, SHARD_THREADS, 0, s>>>(S, tokens, lens, c, B, K, stats, status);
-    } else {
-        if (shard_vec<float>(sh)) shard_stats_kernel<float, true><<<grid, SHARD_THREADS, 0, s>>>(S, tokens, lens, c, B, K, stats, status);
-        else shard_stats_kernel<float, false><<<grid, SHARD_THREADS, 0, s>>>(S, tokens, lens, c, B, K, stats, status);
-    }
+    if (sh.dtype == SPECDEC_BF16) launch_stats_t<__nv_bfloat16>(sh, S, tokens, lens, c, B, K, stats, status, s);
+    else launch_stats_t<float>(sh, S, tokens, lens, c, B, K, stats, status, s);
     return cudaGetLastError();
 }
 
