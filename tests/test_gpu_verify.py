@@ -257,3 +257,24 @@ def test_wide_shapes(ctx, flags):
         gpu = parity.run_gpu_verify(ctx, inp, flags)
         rep = parity.classify_rows(inp, gpu, dtype="f32")
         assert rep["rows"] == B and ctx.device_status() == 0
+
+
+@pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
+def test_many_candidates_per_row(flags):
+    """K = 80: more positions than one ballot word or the fused kernel's six-bit row record hold."""
+    c = specdec.Context(max_B=4, max_K=80)
+    cfg = wl.Workload("k80", B=4, K=80, V=2048, dtype="bf16", sigma_d=2.0, sigma_n=0.3, T=1.0, ragged=True, seed=80)
+    inp = wl.make_verify_inputs(cfg, threads=1)
+    inp["cand_len"][:] = [80, 79, 33, 64]
+    inp = dict(inp)
+    # regenerate the rows for the forced lengths so that unread rows stay poisoned consistently
+    for b in range(4):
+        t, d, y = wl._row_logits(cfg, b, int(inp["cand_len"][b]), cfg.sigma_n, False)
+        inp["target_logits"][b], inp["draft_logits"][b], inp["cand_tokens"][b] = t, d, y
+    inp["draft_logits"][0] = inp["target_logits"][0][:80]      # p = q on row 0: all 80 candidates are accepted
+    inp["draft_logits"][3, :40] = inp["target_logits"][3, :40]  # row 3 gets past the first ballot word at least
+    gpu = parity.run_gpu_verify(c, inp, flags)
+    rep = parity.classify_rows(inp, gpu, dtype="f32")
+    assert rep["rows"] == 4 and c.device_status() == 0
+    assert gpu["n_accepted"][0] == 80 and gpu["n_accepted"][3] >= 40
+    c.close()
