@@ -62,7 +62,11 @@ typedef enum {
 #define SPECDEC_VERIFY_STREAM  2u /* persistent CTAs fed by bulk async copies (TMA): one launch for the
                                     statistics and accept tests, a second for the draws           */
 #define SPECDEC_VERIFY_FUSED   3u /* the same pipeline in one launch: CTAs that run out of units
-                                    stream the draws of rows that are already resolved             */
+                                    stream the draws of rows that are already resolved.  Its CTAs
+                                    wait (bounded) for rows resolved by other CTAs of the launch, so
+                                    it needs the GPU to itself: if another process or stream keeps
+                                    some of its CTAs from being resident, waits can run out, the
+                                    call reports SPECDEC_DATA_WAIT_LIMIT and its outputs are invalid */
 #define SPECDEC_VERIFY_CLUSTER 4u /* small batches: a cluster of 2-8 CTAs per (row, position), each taking
                                     a slice of the vocabulary, combined through distributed shared
                                     memory; picked automatically while the units fit the SMs twice   */
@@ -276,7 +280,8 @@ int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const specdec_head
  * Threshold stop rule (Section 4.3; loop of Algorithm 1): for each row the first 0-based
  * position j with 1 - prod_{i<=j} accept_prob[b,i] > h (strict), scanning i < cand_len[b]
  * (K when cand_len is NULL).  stop_pos[b] = j, or cand_len[b] (resp. K) if the rule never
- * fires.  Products are formed sequentially in fp32.
+ * fires.  Products are formed sequentially in fp32.  A cand_len[b] outside [0, K] gives
+ * stop_pos[b] = -1 and sets SPECDEC_DATA_BAD_LENGTH in the device status word; the row is not read.
  *   accept_prob dev [B, K] f32, cand_len dev [B] int32 or NULL, stop_pos dev out [B] int32
  */
 int specdec_stop(specdec_ctx* ctx, const float* accept_prob, const int32_t* cand_len,

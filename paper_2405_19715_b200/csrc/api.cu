@@ -31,14 +31,6 @@ int cuda_fail(specdec_ctx* ctx, cudaError_t e, const char* what) {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// Every entry point runs on the context's GPU, whichever device the calling thread had current.
-int use_device(specdec_ctx* ctx) {
-    int cur = -1;
-    if (cudaGetDevice(&cur) == cudaSuccess && cur == ctx->device) return SPECDEC_OK;   // the usual case, no driver call
-    cudaError_t e = cudaSetDevice(ctx->device);
-    return e == cudaSuccess ? SPECDEC_OK : cuda_fail(ctx, e, "cudaSetDevice");
-}
-
 int check_verify_args(specdec_ctx* ctx, const void* target, const void* draft, int dtype, const int32_t* tokens,
                       const float* uniforms, float T, int B, int K, int V, const int32_t* n_acc,
                       const int32_t* next, uint32_t flags) {
@@ -52,10 +44,18 @@ int check_verify_args(specdec_ctx* ctx, const void* target, const void* draft, i
     if (B > ctx->max_B || K > ctx->max_K)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: B=%d K=%d exceed the context (max_B=%d max_K=%d)", B, K, ctx->max_B, ctx->max_K);
     if (V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: V=%d above 2^22", V);
-    return use_device(ctx);
+    return specdec_use_device(ctx);
 }
 
 }  // namespace
+
+// Every entry point runs on the context's GPU, whichever device the calling thread had current.
+int specdec_use_device(specdec_ctx* ctx) {
+    int cur = -1;
+    if (cudaGetDevice(&cur) == cudaSuccess && cur == ctx->device) return SPECDEC_OK;   // the usual case, no driver call
+    cudaError_t e = cudaSetDevice(ctx->device);
+    return e == cudaSuccess ? SPECDEC_OK : cuda_fail(ctx, e, "cudaSetDevice");
+}
 
 extern "C" {
 
@@ -128,7 +128,7 @@ uint64_t specdec_launch_count(const specdec_ctx* ctx) { return ctx ? ctx->launch
 
 int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits) {
     if (!ctx) return SPECDEC_EINVAL;
-    if (int rc = use_device(ctx)) return rc;
+    if (int rc = specdec_use_device(ctx)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint32_t host = 0;
     CU(ctx, cudaMemcpyAsync(&host, ctx->status, sizeof(host), cudaMemcpyDeviceToHost, s));
@@ -262,7 +262,7 @@ int specdec_sample(specdec_ctx* ctx, const void* logits, specdec_dtype dtype, co
     if (B < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "sample: B and V must be >= 1 (got %d, %d)", B, V);
     if (B > ctx->max_B) return fail(ctx, SPECDEC_EUNSUPPORTED, "sample: B=%d exceeds the context (max_B=%d)", B, ctx->max_B);
     if (top_k > 256 && top_k < V) return fail(ctx, SPECDEC_EINVAL, "sample: top_k must be <= 256, or <= 0 / >= V for none (got %d)", top_k);
-    if (int rc0 = use_device(ctx)) return rc0;
+    if (int rc0 = specdec_use_device(ctx)) return rc0;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     ctx->epoch = (ctx->epoch + 1) & 0x3fffffffu;
     if ((ctx->epoch & 0xffffffu) == 0)
@@ -310,7 +310,7 @@ int check_shard_args(specdec_ctx* ctx, const specdec_shard* sh, float T, int B, 
         return fail(ctx, SPECDEC_EINVAL, "%s: columns [%d, %d + %d) do not lie in a vocabulary of %d", who, sh->v_offset, sh->v_offset, sh->V_shard, sh->V);
     if (!(T > 0.f) || !std::isfinite(T)) return fail(ctx, SPECDEC_EINVAL, "%s: temperature must be positive and finite", who);
     if (sh->V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "%s: V=%d above 2^22", who, sh->V);
-    return use_device(ctx);
+    return specdec_use_device(ctx);
 }
 }  // namespace
 
@@ -374,6 +374,8 @@ int specdec_verify_greedy(specdec_ctx* ctx, const void* target_logits, specdec_d
     if (B < 1 || K < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "verify_greedy: B, K, V must be >= 1");
     if (B > ctx->max_B || K > ctx->max_K)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_greedy: B=%d K=%d exceed the context (max_B=%d max_K=%d)", B, K, ctx->max_B, ctx->max_K);
+    if (V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_greedy: V=%d above 2^22", V);
+    if (int rc = specdec_use_device(ctx)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     ctx->epoch = (ctx->epoch + 1) & 0x3fffffffu;
     if ((ctx->epoch & 0xffffffu) == 0)
@@ -457,8 +459,8 @@ int specdec_stop(specdec_ctx* ctx, const float* accept_prob, const int32_t* cand
     if (!accept_prob || !stop_pos) return fail(ctx, SPECDEC_EINVAL, "stop: null pointer argument");
     if (B < 1 || K < 1) return fail(ctx, SPECDEC_EINVAL, "stop: B and K must be >= 1");
     if (h != h) return fail(ctx, SPECDEC_EINVAL, "stop: threshold is NaN");
-    if (int rc = use_device(ctx)) return rc;
-    cudaError_t e = launch_stop(accept_prob, cand_len, h, B, K, stop_pos, static_cast<cudaStream_t>(stream));
+    if (int rc = specdec_use_device(ctx)) return rc;
+    cudaError_t e = launch_stop(accept_prob, cand_len, h, B, K, stop_pos, ctx->status, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "stop launch");
     ctx->launches += 1;
     return SPECDEC_OK;
@@ -470,7 +472,7 @@ int specdec_stop_step(specdec_ctx* ctx, const float* accept_prob_step, float* p_
     if (!accept_prob_step || !p_hat || !stop) return fail(ctx, SPECDEC_EINVAL, "stop_step: null pointer argument");
     if (B < 1) return fail(ctx, SPECDEC_EINVAL, "stop_step: B must be >= 1");
     if (h != h) return fail(ctx, SPECDEC_EINVAL, "stop_step: threshold is NaN");
-    if (int rc = use_device(ctx)) return rc;
+    if (int rc = specdec_use_device(ctx)) return rc;
     cudaError_t e = launch_stop_step(accept_prob_step, p_hat, h, B, stop, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "stop_step launch");
     ctx->launches += 1;
@@ -479,7 +481,7 @@ int specdec_stop_step(specdec_ctx* ctx, const float* accept_prob_step, float* p_
 
 int specdec_selftest_wait_limit(specdec_ctx* ctx, void* stream) {
     if (!ctx) return SPECDEC_EINVAL;
-    if (int rc = use_device(ctx)) return rc;
+    if (int rc = specdec_use_device(ctx)) return rc;
     cudaError_t e = launch_wait_limit_selftest(ctx->status, static_cast<cudaStream_t>(stream));
     if (e != cudaSuccess) return cuda_fail(ctx, e, "selftest launch");
     ctx->launches += 1;

@@ -639,9 +639,7 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
         return fail(ctx, SPECDEC_EUNSUPPORTED, "accept_head: B*K or d exceed the context");
     if (reinterpret_cast<uintptr_t>(hidden) % 16 != 0 || reinterpret_cast<uintptr_t>(head->w_out) % 16 != 0)
         return fail(ctx, SPECDEC_EINVAL, "accept_head: hidden and w_out must be 16-byte aligned");
-    int cur_dev = -1;
-    if ((cudaGetDevice(&cur_dev) != cudaSuccess || cur_dev != ctx->device) && cudaSetDevice(ctx->device) != cudaSuccess)
-        return fail(ctx, SPECDEC_ECUDA, "accept_head: cudaSetDevice failed");
+    if (int rc = specdec_use_device(ctx)) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(hidden);
     if (D == 0) {

@@ -56,6 +56,9 @@ struct VerifyParams {
     uint32_t epoch;
 };
 
+// Makes the context's GPU the calling thread's current device (api.cu); SPECDEC_OK or SPECDEC_ECUDA.
+int specdec_use_device(specdec_ctx* ctx);
+
 // Launchers (verify.cu, verify_stream.cu, stop.cu, head.cu).  Return a cudaError_t.
 cudaError_t launch_verify_direct(const VerifyParams& p, specdec_dtype dtype, cudaStream_t s, int* n_launch);
 cudaError_t launch_verify_stream(const VerifyParams& p, specdec_dtype dtype, int sm_count, cudaStream_t s,
@@ -65,7 +68,7 @@ cudaError_t launch_verify_fused(const VerifyParams& p, specdec_dtype dtype, int 
 bool verify_stream_supported(const VerifyParams& p, specdec_dtype dtype);
 cudaError_t launch_greedy(const VerifyParams& p, specdec_dtype dtype, int32_t* argmax_out, cudaStream_t s);
 cudaError_t launch_stop(const float* accept_prob, const int32_t* lens, float h, int B, int K,
-                        int32_t* stop_pos, cudaStream_t s);
+                        int32_t* stop_pos, uint32_t* status, cudaStream_t s);
 cudaError_t launch_stop_step(const float* accept_prob_step, float* p_hat, float h, int B, int32_t* stop,
                              cudaStream_t s);
 cudaError_t launch_wait_limit_selftest(uint32_t* status, cudaStream_t s);

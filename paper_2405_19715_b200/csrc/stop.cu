@@ -5,11 +5,15 @@
 namespace {
 
 __global__ void stop_kernel(const float* __restrict__ a, const int32_t* __restrict__ lens, float h, int B, int K,
-                            int32_t* __restrict__ stop_pos) {
+                            int32_t* __restrict__ stop_pos, uint32_t* __restrict__ status) {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
-    int L = lens ? lens[b] : K;
-    L = L < 0 ? 0 : (L > K ? K : L);
+    const int L = lens ? lens[b] : K;
+    if (L < 0 || L > K) {                        // bad length: the row reports -1, nothing is read
+        atomicOr(status, SPECDEC_DATA_BAD_LENGTH);
+        stop_pos[b] = -1;
+        return;
+    }
     const float* row = a + (size_t)b * K;
     float c = 1.f;
     int pos = L;
@@ -39,8 +43,8 @@ cudaError_t launch_stop_step(const float* accept_prob_step, float* p_hat, float 
 }
 
 cudaError_t launch_stop(const float* accept_prob, const int32_t* lens, float h, int B, int K, int32_t* stop_pos,
-                        cudaStream_t s) {
+                        uint32_t* status, cudaStream_t s) {
     const int threads = 128;
-    stop_kernel<<<(B + threads - 1) / threads, threads, 0, s>>>(accept_prob, lens, h, B, K, stop_pos);
+    stop_kernel<<<(B + threads - 1) / threads, threads, 0, s>>>(accept_prob, lens, h, B, K, stop_pos, status);
     return cudaGetLastError();
 }

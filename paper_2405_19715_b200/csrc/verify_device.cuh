@@ -338,6 +338,14 @@ struct Unit {
     bool bonus;                // i == L: the p_{L+1} row, no draft
 };
 
+// p(y) / q(y) from the two base-2 log-probabilities.  p(y) = 0 (a masked target logit) is a certain
+// rejection whatever q(y) is -- also when both are zero, where the difference of the logs is not a
+// number; q(y) = 0 < p(y) gives +inf (always accepted).
+__device__ __forceinline__ float ratio_from_logs(float lp, float lq) {
+    const float ratio = exp2f(lp - lq);
+    return (lp == -INFINITY || ratio != ratio) ? 0.f : ratio;
+}
+
 // Accept test of one unit, called by one full warp once the unit's statistics are known (they
 // only need to be valid in lane 0, as do t_y, d_y, y_ok and r = uniforms[b, i]): optional
 // outputs and flag publication.  Returns the flag state (0 for the bonus unit) in every lane.
@@ -354,7 +362,7 @@ __device__ __forceinline__ int unit_accept(const VerifyParams& P, const Unit& u,
             // against the same rs the sum was accumulated with.
             const float lp = fmaf(t_y, P.c, -ap.rs) - log2f(ap.s);
             const float lq = fmaf(d_y, P.c, -aq.rs) - log2f(aq.s);
-            const float ratio = exp2f(lp - lq);
+            const float ratio = ratio_from_logs(lp, lq);
             state = !y_ok ? FLAG_BAD : (r >= ratio ? FLAG_REJECT : FLAG_ACCEPT);   // r == ratio rejects
             if (!y_ok) atomicOr(P.status, SPECDEC_DATA_BAD_TOKEN);
             if (P.ratio) P.ratio[(size_t)u.b * K + u.i] = y_ok ? fminf(1.f, ratio) : -1.f;

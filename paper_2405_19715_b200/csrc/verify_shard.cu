@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(32) shard_accept_kernel(const float* __restric
             const Merged m = merge_records(stats_all, n_shards, B, K, b, i);
             const float lp = fmaf(m.t_y, c, -m.p.rs) - log2f(m.p.s);
             const float lq = fmaf(m.d_y, c, -m.q.rs) - log2f(m.q.s);
-            const float ratio = exp2f(lp - lq);
+            const float ratio = ratio_from_logs(lp, lq);
             const bool ok = m.owned == 1.f;          // exactly one rank held column y
             const float r = uniforms[(size_t)b * (K + 1) + i];
             state = !ok ? FLAG_BAD : (r >= ratio ? FLAG_REJECT : FLAG_ACCEPT);     // r == ratio rejects

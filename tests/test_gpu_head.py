@@ -138,6 +138,37 @@ def test_config5_head_stop_verify_chain():
     ctx.close()
 
 
+def test_head_at_the_benchmark_shape():
+    """The shape the benchmark times: B*K = 4096 rows (cfg4's 256 x 16 positions), d = 4096, D = 2 of
+    the cfg5 recipe, i.e. 512 tiles of 128 x 256 on 148 persistent CTAs (3.46 tiles per CTA).  All 4096
+    outputs against the oracle; repeatable bit for bit."""
+    cfg = wl.CONFIGS["cfg5"].scaled(B=256, K=16)
+    ctx = specdec.Context(cfg.B, cfg.K, max_d=cfg.d)
+    hd = wl.make_head_inputs(cfg)
+    Ws = [w for w, _ in hd["blocks"]]
+    bs = [b for _, b in hd["blocks"]]
+    got = _run_head(ctx, hd["hidden"], Ws, bs, hd["w_out"], float(hd["b_out"]))
+    want = orc.accept_head(hd["hidden"], hd["blocks"], hd["w_out"], float(hd["b_out"]))
+    err = np.abs(got - want) / want
+    print("head 4096 x 4096 x 2 max rel err", err.max())
+    assert got.shape == (256, 16) and err.max() <= HEAD_RTOL and want.std() > 1e-2
+    assert np.array_equal(got, _run_head(ctx, hd["hidden"], Ws, bs, hd["w_out"], float(hd["b_out"])))
+    ctx.close()
+
+
+@pytest.mark.parametrize("rows", [17, 32, 33, 64, 65, 128, 129, 200, 256])
+def test_head_up_to_256_rows_at_full_width(rows):
+    """17 to 256 rows at d = 4096, D = 2 (Eq. 3 once per drafted token for that many sequences)."""
+    ctx = specdec.Context(rows, 1, max_d=4096)
+    hidden, Ws, bs, w_out, b_out = _head_problem(900 + rows, rows, 1, 4096, 2, True, std=0.02)
+    got = _run_head(ctx, hidden, Ws, bs, w_out, b_out)
+    want = orc.accept_head(hidden, list(zip(Ws, bs)), w_out, b_out)
+    err = np.abs(got - want) / want
+    assert err.max() <= HEAD_RTOL, (err.max(), np.argmax(err))
+    assert np.array_equal(got, _run_head(ctx, hidden, Ws, bs, w_out, b_out))
+    ctx.close()
+
+
 def test_online_head_and_stop_step_replay_algorithm_1():
     """Algorithm 1's loop, one drafted token per call: head on [B,1,d] (narrow-tile GEMM), then
     specdec_stop_step.  Each step is checked against the oracle; the replay must also reproduce the

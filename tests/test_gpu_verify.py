@@ -7,6 +7,7 @@ pytestmark = pytest.mark.gpu
 
 from paper_2405_19715_b200 import specdec, workloads as wl  # noqa: E402
 from tests import parity  # noqa: E402
+from oracle.specdec_oracle import stop_rule as orc_stop  # noqa: E402
 
 KERNELS = [specdec.VERIFY_DIRECT, specdec.VERIFY_STREAM, specdec.VERIFY_FUSED, specdec.VERIFY_CLUSTER]
 KERNEL_IDS = ["direct", "stream", "fused", "cluster"]
@@ -70,31 +71,27 @@ def test_configs_1_to_3(ctx, name, flags):
         assert np.array_equal(gpu[k], gpu2[k]), k
 
 
-@pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
-def test_config4_full_size_sampled_rows(ctx, flags):
-    """Full-size cfg4 (B=256, K=16, V=128256, bf16) in the launch configuration the benchmark times;
-    the oracle checks a sample of rows (peaked and ordinary) one by one, properties cover the rest."""
+@pytest.fixture(scope="module")
+def cfg4_problem():
+    """cfg4's inputs and the oracle's answer for every one of its 256 rows, made once for all kernels."""
     cfg = wl.CONFIGS["cfg4"]
     inp = wl.make_verify_inputs(cfg)
+    return cfg, inp, parity.oracle_rows(inp)
+
+
+@pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
+def test_config4_full_size_every_row(ctx, cfg4_problem, flags):
+    """Full-size cfg4 (B=256, K=16, V=128256, bf16) in the launch configuration the benchmark times:
+    every row's n, y', accept ratios, p(y), q(y), normalisers and residual mass against the oracle."""
+    cfg, inp, oracle_out = cfg4_problem
     gpu = parity.run_gpu_verify(ctx, inp, flags)
     assert ctx.device_status() == 0
-    peaked = np.nonzero(inp["peaked"])[0]
-    plain = np.nonzero(~inp["peaked"])[0]
-    rows = list(peaked[:3]) + list(plain[:5]) + [int(plain[-1])]
-    rep = parity.classify_rows(inp, gpu, rows=rows, dtype="f32")
-    print("cfg4", rep)
-    n, tok = gpu["n_accepted"], gpu["next_token"]
-    assert np.all((n >= 0) & (n <= cfg.K)) and np.all((tok >= 0) & (tok < cfg.V))
+    rep = parity.classify_rows(inp, gpu, dtype="f32", oracle_out=oracle_out)
+    print("cfg4", KERNEL_IDS[KERNELS.index(flags)], rep)
+    assert rep["rows"] == cfg.B and rep["exact"] + rep["boundary_n"] + rep["boundary_token"] == cfg.B
     # rows whose drafted tokens carry +12 on the target are accepted almost surely
-    assert (n[peaked] == cfg.K).mean() > 0.8
-    # accept ratios decide n: first position with r >= ratio
-    r = inp["uniforms"][:, :cfg.K]
-    rej = r >= gpu["accept_ratio"]
-    first = np.where(rej.any(1), rej.argmax(1), cfg.K)
-    assert np.array_equal(first, n)
-    # the drawn token has positive residual weight: p(y') > q(y') needs the logits only up to lse,
-    # checked on the sampled rows by the oracle; here every row's mass is within (0, 1]
-    assert np.all((gpu["resid_mass"] > 0) & (gpu["resid_mass"] <= 1.0 + 1e-5))
+    peaked = np.nonzero(inp["peaked"])[0]
+    assert (gpu["n_accepted"][peaked] == cfg.K).mean() > 0.8
 
 
 @pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
@@ -132,6 +129,14 @@ def test_special_cases(ctx, flags):
     gpu = parity.run_gpu_verify(ctx, masked, flags)
     parity.classify_rows(masked, gpu, dtype="f32")
     assert np.all(gpu["next_token"] >= 100)
+    # a drafted token masked in both rows: p(y) = q(y) = 0 is a certain rejection, y' never lands on it
+    t5, d5 = t.copy(), d.copy()
+    for b in range(B):
+        t5[b, 2, y[b, 2]] = d5[b, 2, y[b, 2]] = -np.inf
+    both = dict(base, target_logits=t5, draft_logits=d5, uniforms=np.zeros_like(u))    # r = 0 accepts any ratio > 0
+    gpu = parity.run_gpu_verify(ctx, both, flags)
+    assert np.all(gpu["n_accepted"] == 2) and np.all(gpu["accept_ratio"][:, 2] == 0.0)
+    parity.classify_rows(both, gpu, dtype="f32")
     # low temperature approaches greedy decoding
     cold = dict(base, target_logits=t + rng.normal(scale=1.0, size=t.shape).astype(np.float32),
                 cand_tokens=d.argmax(-1).astype(np.int32), temperature=np.float32(0.05))
@@ -224,6 +229,14 @@ def test_stop_rule_parity(ctx):
             pos = specdec.specdec_stop(ctx, ta, h, tl).cpu().numpy()
             rep = parity.classify_stop(a, h, pos, lens)
             assert rep["exact"] + rep["boundary"] == cfg.B
+    # a candidate length outside [0, K] gives -1 for that row only and sets the status bit
+    a = np.random.default_rng(2).uniform(0.5, 1.0, size=(5, 6)).astype(np.float32)
+    lens = np.array([6, 7, 3, -1, 0], np.int32)
+    pos = specdec.specdec_stop(ctx, torch.from_numpy(a).cuda(), 0.4, torch.from_numpy(lens).cuda()).cpu().numpy()
+    assert ctx.device_status() == specdec.DATA_BAD_LENGTH and ctx.device_status() == 0
+    assert pos[1] == -1 and pos[3] == -1
+    good = [0, 2, 4]
+    assert np.array_equal(pos[good], orc_stop(a[good], 0.4, lens[good]))
     # thresholds outside (0,1) and rows of ones
     a = np.ones((4, 7), np.float32)
     assert np.all(specdec.specdec_stop(ctx, torch.from_numpy(a).cuda(), 0.0).cpu().numpy() == 7)

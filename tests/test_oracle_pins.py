@@ -493,6 +493,66 @@ def test_greedy_case_is_the_low_temperature_limit():
     assert np.array_equal(cold["n_accepted"], n_g) and np.array_equal(cold["next_token"], tok_g)
 
 
+def test_greedy_ragged_lengths_equal_the_truncated_problem():
+    """Section 4.1 on a ragged batch: a row of candidate length L is the K = L problem of its first
+    L positions; rows of the target beyond position L are never looked at (they are poisoned with NaN
+    here and must not change anything) and report -1 in target_argmax.  The expected values come from
+    torch.argmax row by row, not from the function under test."""
+    rng = np.random.default_rng(21)
+    B, K, V = 9, 6, 17
+    t = rng.normal(scale=2, size=(B, K + 1, V)).astype(np.float32)
+    am_full = torch.from_numpy(t).double().argmax(-1).numpy()
+    lens = np.array([0, 1, 2, 3, 4, 5, 6, 3, 6], np.int32)
+    y = am_full[:, :K].astype(np.int32).copy()                 # all candidates match ...
+    y[4, 2] = (y[4, 2] + 1) % V                                # ... except row 4 at position 2 (< L = 4)
+    y[7, 3] = (y[7, 3] + 1) % V                                # row 7: mismatch at position 3 = L: not a candidate
+    y[8, 0] = (y[8, 0] + 1) % V                                # row 8: first position mismatches
+    tp, yp = t.copy(), y.copy()
+    for b in range(B):
+        tp[b, lens[b] + 1:] = np.nan
+        yp[b, lens[b]:] = -7
+    n, tok, am = orc.greedy_verify_tokens(tp, yp, lens)
+    assert n.tolist() == [0, 1, 2, 3, 2, 5, 6, 3, 0]
+    for b in range(B):
+        assert tok[b] == am_full[b, n[b]]
+        assert np.array_equal(am[b, :lens[b] + 1], am_full[b, :lens[b] + 1]) and np.all(am[b, lens[b] + 1:] == -1)
+        # the truncated problem: K = L, no cand_len argument
+        L = int(lens[b])
+        if L >= 1:
+            n1, tok1, _ = orc.greedy_verify_tokens(t[b:b + 1, :L + 1], y[b:b + 1, :L], None)
+            assert (n1[0], tok1[0]) == (n[b], tok[b])
+    # ties resolve to the lowest index
+    tie = np.zeros((1, 2, 5), np.float32)
+    tie[0, 0, [1, 3]] = 2.0
+    n, tok, am = orc.greedy_verify_tokens(tie, np.array([[3]], np.int32), np.array([1], np.int32))
+    assert (n[0], tok[0], am[0].tolist()) == (0, 1, [1, 0])
+
+
+def test_drafted_token_with_zero_probability_under_both_models_is_rejected():
+    """p(y) = q(y) = 0 (the logit of y is -inf in both rows): the ratio of the accept test is read as
+    0, a certain rejection, as for any p(y) = 0; y' then comes from the residual, which gives y no
+    weight.  Expected values from scipy's softmax and the probability-level core."""
+    rng = np.random.default_rng(8)
+    K, V = 3, 11
+    d = rng.normal(scale=2, size=(1, K, V)).astype(np.float32)
+    t = np.concatenate([d, d[:, :1]], 1) + rng.normal(size=(1, K + 1, V)).astype(np.float32)
+    y = np.array([[2, 5, 7]], np.int32)
+    t[0, 1, 5] = d[0, 1, 5] = -np.inf
+    t[0, 0] = d[0, 0]                                          # position 0: p = q, accepted for any r < 1
+    u = np.array([[0.999, 0.0, 0.5, 0.3]], np.float32)         # r_1 = 0 would accept any positive ratio
+    o = orc.verify_correct(t, d, y, None, u, 1.0)
+    assert o["n_accepted"][0] == 1 and o["accept_ratio"][0, 1] == 0.0 and o["p_y"][0, 1] == 0.0
+    p = scipy.special.softmax(t[0].astype(np.float64), axis=-1)
+    q = scipy.special.softmax(d[0].astype(np.float64), axis=-1)
+    n, tok, ratios, W = orc.verify_from_probs(p, q, y[0], K, u[0, :K].astype(np.float64), float(u[0, K]))
+    assert (n, tok) == (1, o["next_token"][0]) and ratios[1] == 0 and tok != 5
+    # q(y) = 0 < p(y): always accepted
+    t2, d2 = t.copy(), d.copy()
+    t2[0, 1, 5] = 0.0
+    o2 = orc.verify_correct(t2, d2, y, None, np.array([[0.999, 0.999, 0.999, 0.3]], np.float32), 1.0)
+    assert o2["accept_ratio"][0, 1] == 1.0 and o2["n_accepted"][0] >= 2
+
+
 # ----------------------------------------------------------------------------- planted mistakes
 def test_pins_catch_planted_mistakes(monkeypatch):
     """Plant typical slips in the oracle (on the CPU) and check the exact-law pin notices."""
