@@ -381,7 +381,7 @@ __global__ void __launch_bounds__(TK_THREADS, 2) verify_topk_kernel(const Verify
             const bool p_in = y_ok && t_y >= tau_p && t_y > -INFINITY, q_in = y_ok && d_y >= tau_q && d_y > -INFINITY;
             if (!p_in) ratio = 0.f;                                      // p'(y) = 0: certain rejection
             else if (!q_in) ratio = INFINITY;
-            else ratio = exp2f((fmaf(t_y, c, -np.hi) - np.lo) - (fmaf(d_y, c, -nq.hi) - nq.lo));
+            else ratio = exp2f(fmaf(t_y, c, -np.rs) - fmaf(d_y, c, -nq.rs)) * (np.inv / nq.inv);
             state = (!y_ok || too_many_ties) ? FLAG_BAD : (r_acc >= ratio ? FLAG_REJECT : FLAG_ACCEPT);
             if (!y_ok) atomicOr(P.status, SPECDEC_DATA_BAD_TOKEN);
             if (P.ratio) P.ratio[(size_t)u.b * P.K + u.i] = state == FLAG_BAD ? -1.f : fminf(1.f, ratio);

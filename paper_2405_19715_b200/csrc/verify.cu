@@ -2,7 +2,7 @@
 // (vectorised where aligned) global loads.  Serves every shape, including rows that are not
 // 16-byte aligned; the streaming kernel in verify_stream.cu is the fast path for large,
 // aligned problems.  Operation: Algorithm 2 of arXiv 2405.19715 (see specdec.h).
-#include "verify_device.cuh"
+#include "verify_unit.cuh"
 
 namespace {
 
@@ -14,80 +14,9 @@ using namespace sd;
 // chain (accept test, draw, row counter) better than a shorter pass does.
 template <typename T, bool VEC, int DIRECT_THREADS>
 __global__ void __launch_bounds__(DIRECT_THREADS, 1024 / DIRECT_THREADS) verify_direct_kernel(const VerifyParams P) {
-    constexpr int N = Elem<T>::EPV;
     extern __shared__ float slab_sum[];
     __shared__ UnitShared sh;
-
-    // position-major unit order: earlier positions of every row are scheduled first, so their
-    // accept flags are usually known by the time a later position decides whether to draw
-    const int unit = blockIdx.x;
-    Unit u;
-    u.i = unit / P.B;
-    u.b = unit - u.i * P.B;
-    u.L = P.lens ? P.lens[u.b] : P.K;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (u.L < 0 || u.L > P.K) {                  // bad length: the row reports -1, nothing is read
-        if (u.i == 0 && tid == 0) {
-            atomicOr(P.status, SPECDEC_DATA_BAD_LENGTH);
-            P.n_acc[u.b] = -1;
-            P.next[u.b] = -1;
-            if (P.rmass) P.rmass[u.b] = 0.f;
-        }
-        return;
-    }
-    if (u.i > u.L) return;
-    u.bonus = (u.i == u.L);
-
-    const size_t V = (size_t)P.V;
-    const T* trow = static_cast<const T*>(P.target) + ((size_t)u.b * (P.K + 1) + u.i) * V;
-    const T* drow = u.bonus ? trow : static_cast<const T*>(P.draft) + ((size_t)u.b * P.K + u.i) * V;
-
-    // everything the accept test needs besides the sums is requested now and arrives during pass 1
-    int y_ok = 1;
-    float t_y = 0.f, d_y = 0.f, r = 0.f;
-    if (tid == 0 && !u.bonus) {
-        r = P.uniforms[(size_t)u.b * (P.K + 1) + u.i];
-        const int y = P.tokens[(size_t)u.b * P.K + u.i];
-        y_ok = (y >= 0 && y < P.V);
-        if (y_ok) { t_y = to_float(trow[y]); d_y = to_float(drow[y]); }
-    }
-
-    // ---- pass 1: softmax statistics of both rows
-    const int nvec = (P.V + N - 1) / N;
-    Acc ap = acc_init(), aq = acc_init();
-    unit_stats<T, VEC, DIRECT_THREADS>(trow, drow, P.V, P.c, u.bonus, tid, ap, aq);
-    ap = warp_merge(ap);
-    aq = warp_merge(aq);
-    if (lane == 0) { sh.wp[warp] = ap; sh.wq[warp] = aq; }
-    __syncthreads();
-    if (warp == 0) {
-        constexpr int NW = DIRECT_THREADS / 32;
-        Acc a = lane < NW ? sh.wp[lane] : acc_init(), b = lane < NW ? sh.wq[lane] : acc_init();
-        a = warp_merge(a);
-        b = warp_merge(b);
-        const int mode = unit_decide(P, u, a, b, t_y, d_y, y_ok, r, lane);
-        if (lane == 0) {
-            sh.np = make_norm(a);
-            sh.nq = u.bonus ? sh.np : make_norm(b);
-            sh.need_draw = mode;
-        }
-    }
-    __syncthreads();
-
-    // ---- pass 2 (only where this position may supply y'): weights, prefix, inverse CDF
-    const int mode = sh.need_draw;
-    if (mode) {
-        const float u01 = P.uniforms[(size_t)u.b * (P.K + 1) + P.K];
-        unit_draw<T, VEC>(P, trow, drow, mode, u01, sh, slab_sum, tid, DIRECT_THREADS, 0);
-        if (mode == 1 && !(sh.total > 1e-30)) {   // p == q to rounding: draw from p itself
-            const double keep = sh.total;
-            __syncthreads();
-            unit_draw<T, VEC>(P, trow, drow, 2, u01, sh, slab_sum, tid, DIRECT_THREADS, 0);
-            if (tid == 0) sh.total = keep;
-            __syncthreads();
-        }
-    }
-    if (warp == 0) unit_finish(P, u, mode != 0, sh.token, mode ? (float)sh.total : 0.f, lane);
+    direct_unit<T, VEC, DIRECT_THREADS>(P, slab_sum, sh);
 }
 
 template <typename T>

@@ -72,8 +72,16 @@ __global__ void __launch_bounds__(CL_THREADS) verify_cluster_kernel(const Verify
     Unit u;
     u.i = unit / P.B;
     u.b = unit - u.i * P.B;
-    u.L = P.lens ? P.lens[u.b] : P.K;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // length, uniform and drafted token are requested together; the drafted token's two logits
+    // right behind the first row loads
+    u.L = P.lens ? ld_early_s32(P.lens + u.b) : P.K;
+    float r = 0.f;
+    int y = 0;
+    if (rank == 0 && tid == 0 && u.i < P.K) {
+        r = ld_early_f32(P.uniforms + (size_t)u.b * (P.K + 1) + u.i);
+        y = ld_early_s32(P.tokens + (size_t)u.b * P.K + u.i);
+    }
     if (u.L < 0 || u.L > P.K) {                    // bad length: the row reports -1, nothing is read
         if (u.i == 0 && rank == 0 && tid == 0) {
             atomicOr(P.status, SPECDEC_DATA_BAD_LENGTH);
@@ -98,26 +106,24 @@ __global__ void __launch_bounds__(CL_THREADS) verify_cluster_kernel(const Verify
     Ps.V = len;
 
     int y_ok = 1;
-    float t_y = 0.f, d_y = 0.f, r = 0.f;
-    if (rank == 0 && tid == 0 && !u.bonus) {
-        r = P.uniforms[(size_t)u.b * (P.K + 1) + u.i];
-        const int y = P.tokens[(size_t)u.b * P.K + u.i];
-        y_ok = (y >= 0 && y < P.V);
-        if (y_ok) { t_y = to_float(trow[y]); d_y = to_float(drow[y]); }
-    }
+    float t_y = 0.f, d_y = 0.f;
+    auto gather_y = [&]() {
+        if (rank == 0 && tid == 0 && !u.bonus) {
+            y_ok = (y >= 0 && y < P.V);
+            if (y_ok) { t_y = ld_early_logit(trow + y); d_y = ld_early_logit(drow + y); }
+        }
+    };
 
     // ---- statistics of the slice
     Acc ap = acc_init(), aq = acc_init();
-    unit_stats<T, VEC, CL_THREADS>(ts, ds, len, P.c, u.bonus, tid, ap, aq);
-    ap = warp_merge(ap);
-    aq = warp_merge(aq);
+    unit_stats<T, VEC, CL_THREADS>(ts, ds, len, P.c, u.bonus, tid, ap, aq, gather_y);
+    warp_merge2(ap, aq);
     if (lane == 0) { sh.wp[warp] = ap; sh.wq[warp] = aq; }
     __syncthreads();
     if (warp == 0) {
         constexpr int NW = CL_THREADS / 32;
         Acc a = lane < NW ? sh.wp[lane] : acc_init(), b = lane < NW ? sh.wq[lane] : acc_init();
-        a = warp_merge(a);
-        b = warp_merge(b);
+        warp_merge2(a, b);
         if (lane == 0) { cs.part_p = a; cs.part_q = b; }
     }
     cl_sync();                                     // every slice's statistics are in place

@@ -246,29 +246,65 @@ __device__ __forceinline__ Acc warp_merge(Acc a) {
     return a;
 }
 
-// log2 of the normaliser as an unevaluated sum hi + lo (fp32 each) so that per-element
-// probabilities 2^(x*c - hi - lo) carry no common scale error.
+// Normaliser of a row: the reference its terms were summed against and the reciprocal of that sum,
+// so that p(x) = 2^(x*c - rs) * inv.  The exponent is formed against the very reference of the
+// sum (no common scale error beyond the rounding of one reciprocal) and nothing needs a logarithm.
 struct Norm {
-    float hi, lo;
+    float rs, inv;
 };
-__device__ __forceinline__ Norm make_norm(const Acc& a) {
-    const double k = (double)a.rs + log2((double)a.s);
-    Norm n;
-    n.hi = (float)k;
-    n.lo = (float)(k - (double)n.hi);
-    return n;
+__device__ __forceinline__ Norm make_norm(const Acc& a) { return Norm{a.rs, 1.f / a.s}; }
+__device__ __forceinline__ float prob(float x, float c, const Norm& n) { return ex2(fmaf(x, c, -n.rs)) * n.inv; }
+
+// CTA-wide merge of per-thread statistics, one warp-level step: both rows' references move to the
+// warp maximum (one redux each), the rescaled sums are added by a butterfly (identical in every lane).
+__device__ __forceinline__ float warp_max(float v) {
+    float m;
+    asm("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(m) : "f"(v));
+    return m;
 }
-__device__ __forceinline__ float prob(float x, float c, const Norm& n) {
-    return ex2(fmaf(x, c, -n.hi) - n.lo);
+__device__ __forceinline__ void warp_merge2(Acc& p, Acc& q) {
+    const float mp = warp_max(p.rs), mq = warp_max(q.rs);
+    float sp = p.s * ex2(p.rs - mp), sq = q.s * ex2(q.rs - mq);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        sp += __shfl_xor_sync(0xffffffffu, sp, o);
+        sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    }
+    p = Acc{mp, sp};
+    q = Acc{mq, sq};
+}
+
+// Loads whose place in the instruction stream matters (operands requested early so that their
+// latency overlaps the streaming pass): the compiler keeps volatile statements in order.
+__device__ __forceinline__ int ld_early_s32(const int32_t* p) {
+    int v;
+    asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float ld_early_f32(const float* p) {
+    float v;
+    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float ld_early_logit(const float* p) { return ld_early_f32(p); }
+__device__ __forceinline__ float ld_early_logit(const __nv_bfloat16* p) {
+    unsigned short v;
+    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return __uint_as_float((uint32_t)v << 16);
 }
 
 // Pass over the two rows of one unit by a CTA of THREADS threads: this thread's share of the
 // softmax statistics (merge with warp_merge / acc_merge).  The draft row is skipped at a bonus
 // position.  VEC: four vectors of each row in flight per thread; the reference is moved from the
 // maximum of the raw inputs, so the exponentials are issued without a data-dependent branch.
-template <typename T, bool VEC, int THREADS>
+struct NoHook {
+    __device__ __forceinline__ void operator()() const {}
+};
+// `after_first_loads` runs once, right after the first round of row loads has been issued and before
+// anything waits for it (the place for a dependent scalar load whose latency should hide there).
+template <typename T, bool VEC, int THREADS, typename Hook = NoHook>
 __device__ __forceinline__ void unit_stats(const T* __restrict__ trow, const T* __restrict__ drow, int V, float c,
-                                           bool bonus, int tid, Acc& ap, Acc& aq) {
+                                           bool bonus, int tid, Acc& ap, Acc& aq, Hook after_first_loads = Hook()) {
     constexpr int N = Elem<T>::EPV;
     const int nvec = (V + N - 1) / N;
     if constexpr (VEC) {
@@ -288,6 +324,7 @@ __device__ __forceinline__ void unit_stats(const T* __restrict__ trow, const T* 
                     if (!bonus) rd[k] = __ldcg(dv + j);
                 }
             }
+            if (j0 == tid) after_first_loads();
             float mt = -INFINITY, md = -INFINITY;
 #pragma unroll
             for (int k = 0; k < U; ++k) {
@@ -309,9 +346,11 @@ __device__ __forceinline__ void unit_stats(const T* __restrict__ trow, const T* 
                 }
             }
         }
+        if (tid >= nvec) after_first_loads();
         ap = acc2_fold(a2);
         aq = acc2_fold(q2);
     } else {
+        after_first_loads();
         float xt[N], xd[N];
         for (int j = tid; j < nvec; j += THREADS) {
             load_vec<T, VEC>(trow, j, V, xt);

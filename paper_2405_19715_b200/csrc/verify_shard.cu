@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(32) shard_accept_kernel(const float* __restric
             const Merged m = merge_records(stats_all, n_shards, B, K, b, n);
             const Norm np = make_norm(m.p), nq = n < L ? make_norm(m.q) : np;
             n_acc[b] = n;
-            *norm_out = make_float4(np.hi, np.lo, nq.hi, nq.lo);
+            *norm_out = make_float4(np.rs, np.inv, nq.rs, nq.inv);
         }
     }
 }

@@ -10,7 +10,7 @@
 #include <cstdio>
 #include <mutex>
 
-#include "verify_device.cuh"
+#include "verify_unit.cuh"
 
 namespace {
 
@@ -35,78 +35,12 @@ uint32_t g_epoch[MAX_DEVICES] = {};
 
 constexpr int STATIC_THREADS = 512;
 
-// Same unit decomposition and arithmetic as the direct kernel (one CTA per (row, position)),
-// without its two-vector unrolling.
+// The unit body of the one-CTA-per-unit kernel, with the fixed array as its scratch.
 template <typename T, bool VEC>
 __global__ void __launch_bounds__(STATIC_THREADS, 2) verify_static_kernel(const VerifyParams P) {
-    constexpr int N = Elem<T>::EPV;
     extern __shared__ float slab_sum[];
     __shared__ UnitShared sh;
-    const int unit = blockIdx.x;
-    Unit u;
-    u.i = unit / P.B;
-    u.b = unit - u.i * P.B;
-    u.L = P.lens ? P.lens[u.b] : P.K;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (u.L < 0 || u.L > P.K) {
-        if (u.i == 0 && tid == 0) {
-            atomicOr(P.status, SPECDEC_DATA_BAD_LENGTH);
-            P.n_acc[u.b] = -1;
-            P.next[u.b] = -1;
-        }
-        return;
-    }
-    if (u.i > u.L) return;
-    u.bonus = (u.i == u.L);
-    const size_t V = (size_t)P.V;
-    const T* trow = static_cast<const T*>(P.target) + ((size_t)u.b * (P.K + 1) + u.i) * V;
-    const T* drow = u.bonus ? trow : static_cast<const T*>(P.draft) + ((size_t)u.b * P.K + u.i) * V;
-    const int nvec = (P.V + N - 1) / N;
-    Acc ap = acc_init(), aq = acc_init();
-    float xt[N], xd[N];
-    for (int j = tid; j < nvec; j += STATIC_THREADS) {
-        load_vec<T, VEC>(trow, j, P.V, xt);
-        acc_update<N>(ap, xt, P.c);
-        if (!u.bonus) {
-            load_vec<T, VEC>(drow, j, P.V, xd);
-            acc_update<N>(aq, xd, P.c);
-        }
-    }
-    ap = warp_merge(ap);
-    aq = warp_merge(aq);
-    if (lane == 0) { sh.wp[warp] = ap; sh.wq[warp] = aq; }
-    __syncthreads();
-    if (warp == 0) {
-        constexpr int NW = STATIC_THREADS / 32;
-        Acc a = lane < NW ? sh.wp[lane] : acc_init(), b = lane < NW ? sh.wq[lane] : acc_init();
-        a = warp_merge(a);
-        b = warp_merge(b);
-        int y = 0, y_ok = 1;
-        float t_y = 0.f, d_y = 0.f, r = 0.f;
-        if (lane == 0 && !u.bonus) {
-            r = P.uniforms[(size_t)u.b * (P.K + 1) + u.i];
-            y = P.tokens[(size_t)u.b * P.K + u.i];
-            y_ok = (y >= 0 && y < P.V);
-            if (y_ok) { t_y = to_float(trow[y]); d_y = to_float(drow[y]); }
-        }
-        const int mode = unit_decide(P, u, a, b, t_y, d_y, y_ok, r, lane);
-        if (lane == 0) {
-            sh.np = make_norm(a);
-            sh.nq = u.bonus ? sh.np : make_norm(b);
-            sh.need_draw = mode;
-        }
-    }
-    __syncthreads();
-    const int mode = sh.need_draw;
-    if (mode) {
-        const float u01 = P.uniforms[(size_t)u.b * (P.K + 1) + P.K];
-        unit_draw<T, VEC>(P, trow, drow, mode, u01, sh, slab_sum, tid, STATIC_THREADS, 0);
-        if (mode == 1 && !(sh.total > 1e-30)) {
-            __syncthreads();
-            unit_draw<T, VEC>(P, trow, drow, 2, u01, sh, slab_sum, tid, STATIC_THREADS, 0);
-        }
-    }
-    if (warp == 0) unit_finish(P, u, mode != 0, sh.token, 0.f, lane);
+    direct_unit<T, VEC, STATIC_THREADS>(P, slab_sum, sh);
 }
 
 int report(char* err, size_t err_len, int code, const char* fmt, ...) {

@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) verify_stream_stats_kernel(
         b = warp_merge(b);
         if (lane == 0) {
             const Norm np = make_norm(a), nq = un.bonus ? np : make_norm(b);
-            P.norms[(size_t)un.b * (P.K + 1) + un.i] = make_float4(np.hi, np.lo, nq.hi, nq.lo);
+            P.norms[(size_t)un.b * (P.K + 1) + un.i] = make_float4(np.rs, np.inv, nq.rs, nq.inv);
         }
         unit_accept(P, un, a, b, t_y, d_y, y_ok, r, lane);
         if (!row_arrive(P, un, lane)) continue;
@@ -742,7 +742,7 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) verify_fused_kernel(const V
         b = warp_merge(b);
         if (lane == 0) {
             const Norm np = make_norm(a), nq = un.bonus ? np : make_norm(b);
-            P.norms[(size_t)un.b * (P.K + 1) + un.i] = make_float4(np.hi, np.lo, nq.hi, nq.lo);
+            P.norms[(size_t)un.b * (P.K + 1) + un.i] = make_float4(np.rs, np.inv, nq.rs, nq.inv);
         }
         unit_accept(P, un, a, b, t_y, d_y, y_ok, r, lane);
         if (!row_arrive(P, un, lane)) continue;

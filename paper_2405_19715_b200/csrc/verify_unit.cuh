@@ -1,0 +1,94 @@
+// One (row, position) unit of verify/correct handled by one CTA (Algorithm 2 of arXiv 2405.19715):
+// the body shared by the one-CTA-per-unit kernel (verify.cu) and the allocation-free entry point's
+// kernel (verify_static.cu), which differ only in where their scratch lives.
+#pragma once
+
+#include "verify_device.cuh"
+
+namespace sd {
+
+// The whole unit: scalar operands requested up front, one streaming pass for the softmax statistics of
+// both rows, accept test, and -- only where this position may supply y' -- a second pass over the
+// same rows for the residual (or bonus) draw; then the row bookkeeping.  `slab_sum` is dynamic shared
+// memory of one float per 32-vector slab of a row.
+template <typename T, bool VEC, int THREADS>
+__device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __restrict__ slab_sum, UnitShared& sh) {
+    // position-major unit order: earlier positions of every row are scheduled first, so their
+    // accept flags are usually known by the time a later position decides whether to draw
+    const int unit = blockIdx.x;
+    Unit u;
+    u.i = unit / P.B;
+    u.b = unit - u.i * P.B;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // Everything the accept test needs besides the sums.  The length, the uniform and the drafted
+    // token are requested together (their addresses do not depend on the length), the two logits of
+    // the drafted token right behind the first row loads: one round trip instead of three in a row.
+    u.L = P.lens ? ld_early_s32(P.lens + u.b) : P.K;
+    float r = 0.f;
+    int y = 0;
+    if (tid == 0 && u.i < P.K) {
+        r = ld_early_f32(P.uniforms + (size_t)u.b * (P.K + 1) + u.i);
+        y = ld_early_s32(P.tokens + (size_t)u.b * P.K + u.i);
+    }
+    if (u.L < 0 || u.L > P.K) {                  // bad length: the row reports -1, nothing is read
+        if (u.i == 0 && tid == 0) {
+            atomicOr(P.status, SPECDEC_DATA_BAD_LENGTH);
+            P.n_acc[u.b] = -1;
+            P.next[u.b] = -1;
+            if (P.rmass) P.rmass[u.b] = 0.f;
+        }
+        return;
+    }
+    if (u.i > u.L) return;
+    u.bonus = (u.i == u.L);
+
+    const size_t V = (size_t)P.V;
+    const T* trow = static_cast<const T*>(P.target) + ((size_t)u.b * (P.K + 1) + u.i) * V;
+    const T* drow = u.bonus ? trow : static_cast<const T*>(P.draft) + ((size_t)u.b * P.K + u.i) * V;
+
+    int y_ok = 1;
+    float t_y = 0.f, d_y = 0.f;
+    auto gather_y = [&]() {
+        if (tid == 0 && !u.bonus) {
+            y_ok = (y >= 0 && y < P.V);
+            if (y_ok) { t_y = ld_early_logit(trow + y); d_y = ld_early_logit(drow + y); }
+        }
+    };
+
+    // ---- pass 1: softmax statistics of both rows
+    Acc ap = acc_init(), aq = acc_init();
+    unit_stats<T, VEC, THREADS>(trow, drow, P.V, P.c, u.bonus, tid, ap, aq, gather_y);
+    warp_merge2(ap, aq);
+    if (lane == 0) { sh.wp[warp] = ap; sh.wq[warp] = aq; }
+    __syncthreads();
+    if (warp == 0) {
+        constexpr int NW = THREADS / 32;
+        Acc a = lane < NW ? sh.wp[lane] : acc_init(), b = lane < NW ? sh.wq[lane] : acc_init();
+        warp_merge2(a, b);
+        const int mode = unit_decide(P, u, a, b, t_y, d_y, y_ok, r, lane);
+        if (lane == 0) {
+            sh.np = make_norm(a);
+            sh.nq = u.bonus ? sh.np : make_norm(b);
+            sh.need_draw = mode;
+        }
+    }
+    __syncthreads();
+
+    // ---- pass 2 (only where this position may supply y'): weights, prefix, inverse CDF
+    const int mode = sh.need_draw;
+    if (mode) {
+        const float u01 = P.uniforms[(size_t)u.b * (P.K + 1) + P.K];
+        unit_draw<T, VEC>(P, trow, drow, mode, u01, sh, slab_sum, tid, THREADS, 0);
+        if (mode == 1 && !(sh.total > 1e-30)) {   // p == q to rounding: draw from p itself
+            const double keep = sh.total;
+            __syncthreads();
+            unit_draw<T, VEC>(P, trow, drow, 2, u01, sh, slab_sum, tid, THREADS, 0);
+            if (tid == 0) sh.total = keep;
+            __syncthreads();
+        }
+    }
+    if (warp == 0) unit_finish(P, u, mode != 0, sh.token, mode ? (float)sh.total : 0.f, lane);
+}
+
+}  // namespace sd

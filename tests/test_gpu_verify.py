@@ -130,10 +130,12 @@ def test_special_cases(ctx, flags):
     parity.classify_rows(masked, gpu, dtype="f32")
     assert np.all(gpu["next_token"] >= 100)
     # a drafted token masked in both rows: p(y) = q(y) = 0 is a certain rejection, y' never lands on it
-    t5, d5 = t.copy(), d.copy()
+    t5, d5 = t + rng.normal(scale=0.8, size=t.shape).astype(np.float32), d.copy()
     for b in range(B):
         t5[b, 2, y[b, 2]] = d5[b, 2, y[b, 2]] = -np.inf
-    both = dict(base, target_logits=t5, draft_logits=d5, uniforms=np.zeros_like(u))    # r = 0 accepts any ratio > 0
+    u5 = u.copy()
+    u5[:, :K] = 0.0                                                                    # r = 0 accepts any ratio > 0
+    both = dict(base, target_logits=t5, draft_logits=d5, uniforms=u5)
     gpu = parity.run_gpu_verify(ctx, both, flags)
     assert np.all(gpu["n_accepted"] == 2) and np.all(gpu["accept_ratio"][:, 2] == 0.0)
     parity.classify_rows(both, gpu, dtype="f32")
