@@ -9,9 +9,9 @@ namespace {
 using namespace sd;
 
 
-// DIRECT_THREADS threads per unit: 512 (two CTAs per SM) when the units fit the machine a few times
-// over, 256 (four per SM) for larger grids, where more resident units hide each unit's dependent
-// chain (accept test, draw, row counter) better than a shorter pass does.
+// DIRECT_THREADS threads per unit: 512 (two CTAs per SM) while the grid fills the machine less than
+// twice, 256 (four per SM) beyond that, where more resident units hide each unit's dependent chain
+// (accept test, draw, row counter) and pack the last wave better than a shorter pass does.
 template <typename T, bool VEC, int DIRECT_THREADS>
 __global__ void __launch_bounds__(DIRECT_THREADS, 1024 / DIRECT_THREADS) verify_direct_kernel(const VerifyParams P) {
     extern __shared__ float slab_sum[];
@@ -33,7 +33,7 @@ cudaError_t launch_t(const VerifyParams& p, cudaStream_t s) {
         if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
         return n;
     }();
-    const bool small_ctas = grid >= 12 * sms;
+    const bool small_ctas = grid >= 4 * sms;
     auto kern = small_ctas ? (vec ? verify_direct_kernel<T, true, 256> : verify_direct_kernel<T, false, 256>)
                            : (vec ? verify_direct_kernel<T, true, 512> : verify_direct_kernel<T, false, 512>);
     if (smem > 40 * 1024) {
