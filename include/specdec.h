@@ -93,6 +93,10 @@ int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits);
 /* Number of kernels this context has launched so far (for launch accounting). */
 uint64_t specdec_launch_count(const specdec_ctx* ctx);
 
+/* Name of the kernel the last specdec_verify_correct / _topk call on this context launched (which
+ * one SPECDEC_VERIFY_AUTO picked): a static string, "none" before the first call. */
+const char* specdec_last_kernel(const specdec_ctx* ctx);
+
 /*
  * Verify and correct one speculation round for B independent rows
  * (Algorithm 2; Algorithm 1 after its drafting loop; rejection step of Appendix C).

@@ -126,6 +126,8 @@ const char* specdec_last_error(const specdec_ctx* ctx) { return ctx ? ctx->err :
 
 uint64_t specdec_launch_count(const specdec_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+const char* specdec_last_kernel(const specdec_ctx* ctx) { return ctx ? ctx->last_kernel : "none"; }
+
 int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits) {
     if (!ctx) return SPECDEC_EINVAL;
     if (int rc = specdec_use_device(ctx)) return rc;
@@ -202,6 +204,10 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
                                                     : launch_verify_direct(p, dtype, s, &n_launch);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "verify_correct launch");
     ctx->launches += n_launch;
+    ctx->last_kernel = kind == SPECDEC_VERIFY_CLUSTER  ? "verify_cluster_kernel"
+                       : kind == SPECDEC_VERIFY_FUSED  ? "verify_fused_kernel"
+                       : kind == SPECDEC_VERIFY_STREAM ? "verify_stream_stats_kernel"
+                                                       : "verify_direct_kernel";
     return SPECDEC_OK;
 }
 
@@ -249,6 +255,7 @@ int specdec_verify_correct_topk(specdec_ctx* ctx, const void* target_logits, con
     cudaError_t e = launch_verify_topk(p, dtype, top_k, s);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "verify_correct_topk launch");
     ctx->launches += 1;
+    ctx->last_kernel = "verify_topk_kernel";
     return SPECDEC_OK;
 }
 

@@ -22,6 +22,7 @@ struct specdec_ctx {
     int32_t* task_ready = nullptr;// [max_B]              fused path: record {epoch:24, mode:2, n:6} of each resolved row
     uint32_t epoch = 0;
     uint64_t launches = 0;
+    const char* last_kernel = "none";   // name of the kernel the last verify/correct call launched
     // staging for the host-buffer entry point (device), grown on demand
     void* stage = nullptr;
     size_t stage_bytes = 0;

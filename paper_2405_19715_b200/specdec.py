@@ -18,7 +18,7 @@ VERIFY_AUTO, VERIFY_DIRECT, VERIFY_STREAM, VERIFY_FUSED, VERIFY_CLUSTER = 0, 1, 
 DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT, DATA_TOPK_TIES = 1, 2, 4, 8
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
-           "specdec_launch_count", "specdec_verify_correct", "specdec_verify_correct_host",
+           "specdec_launch_count", "specdec_last_kernel", "specdec_verify_correct", "specdec_verify_correct_host",
            "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step", "specdec_selftest_wait_limit", "specdec_verify_correct_topk", "specdec_sample",
            "specdec_shard_stats", "specdec_shard_accept", "specdec_shard_draw"]
 SHARD_STATS_WIDTH, SHARD_MAX_RANKS = 8, 64
@@ -59,6 +59,8 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
     lib.specdec_device_status.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint32)]
     lib.specdec_launch_count.argtypes = [C.c_void_p]
     lib.specdec_launch_count.restype = C.c_uint64
+    lib.specdec_last_kernel.argtypes = [C.c_void_p]
+    lib.specdec_last_kernel.restype = C.c_char_p
     lib.specdec_verify_correct.argtypes = [C.c_void_p, vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int, C.c_int,
                                            C.c_int, ip, ip, fp, fp, fp, C.c_uint32, C.c_void_p]
     lib.specdec_verify_correct_host.argtypes = [C.c_void_p, vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int,
@@ -151,6 +153,9 @@ class Context:
 
     def launch_count(self) -> int:
         return int(self.lib.specdec_launch_count(self.handle))
+
+    def last_kernel(self) -> str:
+        return self.lib.specdec_last_kernel(self.handle).decode()
 
     def device_status(self, stream=None) -> int:
         """Synchronises the stream; returns the SPECDEC_DATA_* bits (0 = clean) and clears them."""

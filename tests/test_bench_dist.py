@@ -46,3 +46,18 @@ def test_two_rank_sharding_and_aggregation():
     assert tok0 == tok1 == own0 + own1             # tokens of the whole job
     assert head0 != head1                          # each rank drew its own rows
     assert len(n0) == len(n1) == 3
+
+
+def test_launcher_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` without a launcher around it: the script starts two ranks on 127.0.0.1,
+    each learns its rank and the world size, and rank 0 prints one line for the whole job."""
+    import json
+    import bench
+    rc, out = bench.launch_ranks(2, ["--gpus", "2", "--stub-step", "--steps", "3"], extra_env={"NCCL_DEBUG": "WARN"})
+    assert rc == 0, out
+    lines = [ln for ln in out.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["stub"] is True
+    assert sorted(map(tuple, line["ranks_seen"])) == [(0, 2), (1, 2)]
+    assert line["tokens_per_step"] == 30.0                        # 10 + 20: summed over the ranks
