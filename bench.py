@@ -518,6 +518,83 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+PHASES = [("CTA start -> length known", 0, 1), ("length known -> first row loads issued", 1, 10),
+          ("first loads issued -> first thread's statistics done", 10, 2), ("statistics done -> CTA merged", 2, 3),
+          ("merged -> accept test + draw decision", 3, 4), ("decision -> seen by the CTA", 4, 5),
+          ("draw: slab sums", 5, 6), ("draw: prefix, slab walk", 6, 7), ("no draw: decision -> arrival", 5, 7),
+          ("arrival counted on the row", 7, 8), ("last arriver: ballot + outputs", 8, 9), ("whole unit", 0, 9)]
+
+
+def run_phases(args, cfg):
+    """Per-phase device timestamps of the one-CTA-per-unit verify/correct kernel on `cfg` (cold inputs): builds
+    and loads the diagnostic library (-DSPECDEC_STAMPS) and prints a markdown table.  Not a benchmark line."""
+    from paper_2405_19715_b200 import build as libbuild, specdec
+    specdec.use_library(libbuild.build(stamps=True))
+    to_torch = specdec.from_numpy
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    inp = wl.make_verify_inputs(cfg)
+    es = 2 if cfg.dtype == "bf16" else 4
+    per_copy = cfg.B * (2 * cfg.K + 1) * cfg.V * es
+    copies = 1 if per_copy > 2 * 126e6 else int(np.ceil(2 * 126e6 / per_copy)) + 1
+    base = {k: to_torch(np.ascontiguousarray(inp[k]), "cpu") for k in ("target_logits", "draft_logits", "cand_tokens", "cand_len", "uniforms")}
+    devs = [{k: v.to(dev) for k, v in base.items()} for _ in range(copies)]
+    ctx = specdec.Context(cfg.B, cfg.K)
+    units = cfg.B * (cfg.K + 1)
+    stamps = torch.zeros(units, specdec.STAMP_SLOTS, 2, dtype=torch.int64, device=dev)
+    n_out = torch.empty(cfg.B, dtype=torch.int32, device=dev)
+    t_out = torch.empty(cfg.B, dtype=torch.int32, device=dev)
+    T = float(inp["temperature"])
+    kernel = args.kernel or specdec.VERIFY_DIRECT
+
+    def call(i):
+        d = devs[i % copies]
+        specdec.specdec_verify_correct(ctx, d["target_logits"], d["draft_logits"], d["cand_tokens"], d["cand_len"],
+                                       d["uniforms"], T, n_out, t_out, flags=kernel)
+    for i in range(max(args.warmup, 3)):
+        call(i)
+    torch.cuda.synchronize()
+    ctx.set_phase_stamps(stamps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    durs = {name: [] for name, _, _ in PHASES}
+    done_at, start_at, ev_ms, span = [], [], [], []
+    for i in range(args.steps):
+        stamps.zero_()
+        e0.record()
+        call(i)
+        e1.record()
+        torch.cuda.synchronize()
+        ev_ms.append(e0.elapsed_time(e1))
+        st = stamps.cpu().numpy()
+        g, c = st[:, :, 0].astype(np.float64), st[:, :, 1].astype(np.float64)
+        live = g[:, 9] > 0
+        t0 = g[live, 0].min()
+        start_at.append(np.sort(g[live, 0] - t0) * 1e-3)
+        done_at.append(np.sort(g[live, 9] - t0) * 1e-3)
+        span.append((g[live, 9].max() - t0) * 1e-3)
+        for name, a, b in PHASES:
+            ok = live & (c[:, a] > 0) & (c[:, b] > 0)
+            if name.startswith("no draw"):
+                ok &= c[:, 6] == 0
+            durs[name].append((g[ok, b] - g[ok, a]) * 1e-3)
+    q = lambda x, p: float(np.percentile(x, p)) if len(x) else float("nan")
+    print(f"workload {cfg.name}: B={cfg.B} K={cfg.K} V={cfg.V} {cfg.dtype}, kernel {ctx.last_kernel()}, {args.steps} cold calls; "
+          f"times in us from the device's globaltimer (resolution {np.min(np.diff(np.unique(st[:, :, 0])))} ns)")
+    print(f"call by CUDA events: mean {1e3 * np.mean(ev_ms):.1f} us; first CTA start -> last unit end: mean {np.mean(span):.1f} us")
+    print("| phase | units per call | median | p10 | p90 | max |\n|---|---|---|---|---|---|")
+    for name, _, _ in PHASES:
+        x = np.concatenate(durs[name])
+        print(f"| {name} | {len(x) // args.steps} | {q(x, 50):.2f} | {q(x, 10):.2f} | {q(x, 90):.2f} | {q(x, 100):.2f} |")
+    sa, da = np.mean(np.stack(start_at), 0), np.mean(np.stack(done_at), 0)
+    n = len(sa)
+    print("| unit rank | started at | finished at |\n|---|---|---|")
+    for f in (0.0, 0.25, 0.5, 0.75, 0.9, 0.97, 1.0):
+        k = min(n - 1, int(round(f * (n - 1))))
+        print(f"| {k + 1} of {n} | {sa[k]:.1f} | {da[k]:.1f} |")
+    ctx.set_phase_stamps(None)
+    ctx.close()
+
+
 def run_vocab_sharded(args, cfg):
     """One batch, its vocabulary split over the ranks: statistics -> all-gather -> accept tests and local
     masses -> all-gather -> draw -> max-reduction (strong scaling: the job is the same at every N)."""
@@ -610,6 +687,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling runs)")
+    ap.add_argument("--phases", action="store_true",
+                    help="print per-phase device timestamps of the one-CTA-per-unit verify/correct kernel (diagnostic build)")
     ap.add_argument("--stub-step", action="store_true", help="launcher self-check: gloo ranks on the CPU, empty step")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.workload]
@@ -625,6 +704,8 @@ def main():
         sys.exit(rc)
     if args.stub_step:
         run_stub(args)
+    elif args.phases:
+        run_phases(args, cfg)
     elif args.vocab_shards:
         run_vocab_sharded(args, cfg)
     else:

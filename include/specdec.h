@@ -98,6 +98,21 @@ uint64_t specdec_launch_count(const specdec_ctx* ctx);
 const char* specdec_last_kernel(const specdec_ctx* ctx);
 
 /*
+ * Diagnostic (no counterpart in the paper): phase timestamps of the one-CTA-per-unit verify/correct
+ * kernel.  Only a library compiled with -DSPECDEC_STAMPS contains the code; any other build returns
+ * SPECDEC_EUNSUPPORTED for a non-NULL buffer.  After this call every specdec_verify_correct on the
+ * context whose B*(K+1) <= units makes each (row, position) unit u = i*B + b write
+ * SPECDEC_STAMP_SLOTS pairs {globaltimer in ns, SM cycle counter} at stamps[(u*SLOTS + slot)*2]:
+ * slot 0 CTA started, 1 candidate length known, 10 first row loads issued, 2 first thread's share of
+ * the statistics pass done, 3 CTA-wide merge done, 4 accept test and draw decision taken, 5 decision
+ * seen by all threads, 6 slab sums of the draw done, 7 draw done, 8 arrival counted on the row,
+ * 9 unit finished.  Slots a unit does not reach keep what the caller put there.  stamps = NULL
+ * switches it off.  The buffer (dev, 16*units*SPECDEC_STAMP_SLOTS bytes) stays the caller's.
+ */
+#define SPECDEC_STAMP_SLOTS 16
+int specdec_set_phase_stamps(specdec_ctx* ctx, uint64_t* stamps, size_t units);
+
+/*
  * Verify and correct one speculation round for B independent rows
  * (Algorithm 2; Algorithm 1 after its drafting loop; rejection step of Appendix C).
  *

@@ -31,14 +31,21 @@ def needs_build() -> bool:
     return any(d.stat().st_mtime > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
+def build(force: bool = False, verbose: bool = False, stamps: bool = False) -> Path:
+    """Regular build: libspecdec.so.  stamps=True: the diagnostic build libspecdec_stamps.so, compiled with
+    -DSPECDEC_STAMPS (phase timestamps inside the verify/correct kernel); it is always rebuilt."""
+    if stamps:
+        return _compile(PKG / "libspecdec_stamps.so", PKG / "_build" / "stamps", ["-DSPECDEC_STAMPS"], verbose)
     if not force and not needs_build():
         return LIB
-    obj_dir = PKG / "_build"
-    obj_dir.mkdir(exist_ok=True)
+    return _compile(LIB, PKG / "_build", [], verbose)
+
+
+def _compile(LIB: Path, obj_dir: Path, defines: list, verbose: bool) -> Path:
+    obj_dir.mkdir(parents=True, exist_ok=True)
     nvcc = _nvcc()
     inc = ["-I", str(ROOT / "include"), "-I", str(CSRC)]
-    extra = ["-Xptxas", "-v"] if verbose else []
+    extra = (["-Xptxas", "-v"] if verbose else []) + defines
     procs = []
     for src in SOURCES:
         cmd = [nvcc, *NVCC_FLAGS, *extra, *inc, "-c", str(CSRC / src), "-o", str(obj_dir / (src + ".o"))]
@@ -59,4 +66,4 @@ def build(force: bool = False, verbose: bool = False) -> Path:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, stamps="--stamps" in sys.argv))

@@ -128,6 +128,19 @@ uint64_t specdec_launch_count(const specdec_ctx* ctx) { return ctx ? ctx->launch
 
 const char* specdec_last_kernel(const specdec_ctx* ctx) { return ctx ? ctx->last_kernel : "none"; }
 
+int specdec_set_phase_stamps(specdec_ctx* ctx, uint64_t* stamps, size_t units) {
+    if (!ctx) return SPECDEC_EINVAL;
+#ifdef SPECDEC_STAMPS
+    ctx->stamps = reinterpret_cast<unsigned long long*>(stamps);
+    ctx->stamps_units = stamps ? units : 0;
+    return SPECDEC_OK;
+#else
+    (void)units;
+    if (!stamps) return SPECDEC_OK;
+    return fail(ctx, SPECDEC_EUNSUPPORTED, "set_phase_stamps: this build of the library carries no timestamp code (build with -DSPECDEC_STAMPS)");
+#endif
+}
+
 int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits) {
     if (!ctx) return SPECDEC_EINVAL;
     if (int rc = specdec_use_device(ctx)) return rc;
@@ -184,6 +197,7 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
     p.task_ctl = ctx->task_ctl;
     p.task_ready = ctx->task_ready;
     p.epoch = ctx->epoch;
+    if (ctx->stamps && (size_t)B * (K + 1) <= ctx->stamps_units) p.stamps = ctx->stamps;
 
     const bool stream_ok = verify_stream_supported(p, dtype);
     uint32_t kind = flags;

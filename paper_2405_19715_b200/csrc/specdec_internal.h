@@ -23,6 +23,8 @@ struct specdec_ctx {
     uint32_t epoch = 0;
     uint64_t launches = 0;
     const char* last_kernel = "none";   // name of the kernel the last verify/correct call launched
+    unsigned long long* stamps = nullptr;   // caller's phase-timestamp buffer (diagnostic builds), or null
+    size_t stamps_units = 0;                // (row, position) units it has room for
     // staging for the host-buffer entry point (device), grown on demand
     void* stage = nullptr;
     size_t stage_bytes = 0;
@@ -55,7 +57,10 @@ struct VerifyParams {
     int32_t* task_ctl;
     int32_t* task_ready;
     uint32_t epoch;
+    unsigned long long* stamps = nullptr;   // phase timestamps, SPECDEC_STAMP_SLOTS {globaltimer ns, SM clock} pairs per unit (diagnostic builds)
 };
+
+
 
 // Makes the context's GPU the calling thread's current device (api.cu); SPECDEC_OK or SPECDEC_ECUDA.
 int specdec_use_device(specdec_ctx* ctx);

@@ -15,6 +15,21 @@ namespace sd {
 constexpr float NEG_BIG = -1.0e30f;      // "no reference yet": any finite logit re-references
 constexpr int FLAG_ACCEPT = 1, FLAG_REJECT = 2, FLAG_BAD = 3;
 
+// Phase timestamp of a unit, written by the calling thread.  Compiled in only with -DSPECDEC_STAMPS (the
+// diagnostic build of the library); the regular build carries no trace of it.
+__device__ __forceinline__ void stamp(const VerifyParams& P, int unit, int slot) {
+#ifdef SPECDEC_STAMPS
+    if (P.stamps) {
+        unsigned long long g;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g));
+        const unsigned long long c = (unsigned long long)clock64();
+        unsigned long long* o = P.stamps + ((size_t)unit * SPECDEC_STAMP_SLOTS + slot) * 2;
+        o[0] = g;
+        o[1] = c;
+    }
+#endif
+}
+
 template <typename T> struct Elem;
 template <> struct Elem<float> { static constexpr int EPV = 4; };           // elements per 16 bytes
 template <> struct Elem<__nv_bfloat16> { static constexpr int EPV = 8; };
@@ -639,11 +654,12 @@ __device__ __forceinline__ double slab_total(const float* __restrict__ slab_sum,
 template <typename T, bool VEC>
 __device__ void unit_draw(const VerifyParams& P, const T* __restrict__ trow, const T* __restrict__ drow, int mode,
                           float u01, UnitShared& sh, float* __restrict__ slab_sum, int tid, int nthreads, int bar_id,
-                          double tau_abs = -1.0) {
+                          double tau_abs = -1.0, int stamp_unit = -1) {
     const int warp = tid >> 5, lane = tid & 31;
     const Norm np = sh.np, nq = sh.nq;
     unit_slabs<T, VEC>(P, trow, drow, mode, np, nq, slab_sum, tid, nthreads);
     bar_sync(bar_id, nthreads);
+    if (tid == 0 && stamp_unit >= 0) stamp(P, stamp_unit, 6);
 
     if (warp == 0) {
         double total;
@@ -686,13 +702,15 @@ __device__ __forceinline__ void row_resolve(const VerifyParams& P, const Unit& u
 // For kernels that draw inside the unit: record the draw, count the arrival, and let the last
 // position of the row to arrive pick n and the draw made at position n.
 __device__ __forceinline__ void unit_finish(const VerifyParams& P, const Unit& u, int have_draw, int token, float mass,
-                                            int lane) {
+                                            int lane, int stamp_unit = -1) {
     const int K = P.K;
     if (lane == 0 && have_draw) {
         st_relaxed(&P.draws[(size_t)u.b * (K + 1) + u.i], token);
         st_relaxed(reinterpret_cast<int32_t*>(&P.draw_mass[(size_t)u.b * (K + 1) + u.i]), __float_as_int(mass));
     }
-    if (!row_arrive(P, u, lane)) return;
+    const bool last = row_arrive(P, u, lane);
+    if (lane == 0 && stamp_unit >= 0) stamp(P, stamp_unit, 8);
+    if (!last) return;
     int n, bad;
     row_resolve(P, u, lane, n, bad);
     if (lane == 0) {

@@ -20,6 +20,9 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
     u.i = unit / P.B;
     u.b = unit - u.i * P.B;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // phase timestamps (diagnostic builds): 0 start, 1 length known, 2 this thread's pass 1 done, 3 CTA merged,
+    // 4 accept test and draw decision, 5 decision seen by the CTA, 6 slab sums, 7 draw done, 8 arrival counted, 9 end
+    if (tid == 0) stamp(P, unit, 0);
 
     // Everything the accept test needs besides the sums.  The length, the uniform and the drafted
     // token are requested together (their addresses do not depend on the length), the two logits of
@@ -42,6 +45,7 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
     }
     if (u.i > u.L) return;
     u.bonus = (u.i == u.L);
+    if (tid == 0) stamp(P, unit, 1);
 
     const size_t V = (size_t)P.V;
     const T* trow = static_cast<const T*>(P.target) + ((size_t)u.b * (P.K + 1) + u.i) * V;
@@ -50,6 +54,7 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
     int y_ok = 1;
     float t_y = 0.f, d_y = 0.f;
     auto gather_y = [&]() {
+        if (tid == 0) stamp(P, unit, 10);        // first round of row loads issued
         if (tid == 0 && !u.bonus) {
             y_ok = (y >= 0 && y < P.V);
             if (y_ok) { t_y = ld_early_logit(trow + y); d_y = ld_early_logit(drow + y); }
@@ -59,9 +64,11 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
     // ---- pass 1: softmax statistics of both rows
     Acc ap = acc_init(), aq = acc_init();
     unit_stats<T, VEC, THREADS>(trow, drow, P.V, P.c, u.bonus, tid, ap, aq, gather_y);
+    if (tid == 0) stamp(P, unit, 2);
     warp_merge2(ap, aq);
     if (lane == 0) { sh.wp[warp] = ap; sh.wq[warp] = aq; }
     __syncthreads();
+    if (tid == 0) stamp(P, unit, 3);
     if (warp == 0) {
         constexpr int NW = THREADS / 32;
         Acc a = lane < NW ? sh.wp[lane] : acc_init(), b = lane < NW ? sh.wq[lane] : acc_init();
@@ -71,15 +78,17 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
             sh.np = make_norm(a);
             sh.nq = u.bonus ? sh.np : make_norm(b);
             sh.need_draw = mode;
+            stamp(P, unit, 4);
         }
     }
     __syncthreads();
+    if (tid == 0) stamp(P, unit, 5);
 
     // ---- pass 2 (only where this position may supply y'): weights, prefix, inverse CDF
     const int mode = sh.need_draw;
     if (mode) {
         const float u01 = P.uniforms[(size_t)u.b * (P.K + 1) + P.K];
-        unit_draw<T, VEC>(P, trow, drow, mode, u01, sh, slab_sum, tid, THREADS, 0);
+        unit_draw<T, VEC>(P, trow, drow, mode, u01, sh, slab_sum, tid, THREADS, 0, -1.0, unit);
         if (mode == 1 && !(sh.total > 1e-30)) {   // p == q to rounding: draw from p itself
             const double keep = sh.total;
             __syncthreads();
@@ -88,7 +97,9 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
             __syncthreads();
         }
     }
-    if (warp == 0) unit_finish(P, u, mode != 0, sh.token, mode ? (float)sh.total : 0.f, lane);
+    if (tid == 0) stamp(P, unit, 7);
+    if (warp == 0) unit_finish(P, u, mode != 0, sh.token, mode ? (float)sh.total : 0.f, lane, unit);
+    if (tid == 0) stamp(P, unit, 9);
 }
 
 }  // namespace sd

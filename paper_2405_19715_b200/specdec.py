@@ -18,11 +18,12 @@ VERIFY_AUTO, VERIFY_DIRECT, VERIFY_STREAM, VERIFY_FUSED, VERIFY_CLUSTER = 0, 1, 
 DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT, DATA_TOPK_TIES = 1, 2, 4, 8
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
-           "specdec_launch_count", "specdec_last_kernel", "specdec_verify_correct", "specdec_verify_correct_host",
+           "specdec_launch_count", "specdec_last_kernel", "specdec_set_phase_stamps", "specdec_verify_correct", "specdec_verify_correct_host",
            "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step", "specdec_selftest_wait_limit", "specdec_verify_correct_topk", "specdec_sample",
            "specdec_shard_stats", "specdec_shard_accept", "specdec_shard_draw"]
 SHARD_STATS_WIDTH, SHARD_MAX_RANKS = 8, 64
 STATIC_MAX_UNITS, STATIC_MAX_V = 16384, 262144
+STAMP_SLOTS = 16
 
 
 class SpecdecError(RuntimeError):
@@ -51,6 +52,7 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
         return _lib
     p = Path(path) if path else _build.build()
     lib = C.CDLL(str(p))
+    lib.path = str(p)
     vp, ip, fp = C.c_void_p, C.c_void_p, C.c_void_p
     lib.specdec_create.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int, C.c_int, C.c_int]
     lib.specdec_destroy.argtypes = [C.c_void_p]
@@ -61,6 +63,7 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
     lib.specdec_launch_count.restype = C.c_uint64
     lib.specdec_last_kernel.argtypes = [C.c_void_p]
     lib.specdec_last_kernel.restype = C.c_char_p
+    lib.specdec_set_phase_stamps.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
     lib.specdec_verify_correct.argtypes = [C.c_void_p, vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int, C.c_int,
                                            C.c_int, ip, ip, fp, fp, fp, C.c_uint32, C.c_void_p]
     lib.specdec_verify_correct_host.argtypes = [C.c_void_p, vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int,
@@ -85,6 +88,13 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
     if path is None:
         _lib = lib
     return lib
+
+
+def use_library(path: str | Path) -> C.CDLL:
+    """Make another build of the library (the diagnostic one) the one new contexts load."""
+    global _lib
+    _lib = load_library(path)
+    return _lib
 
 
 def _ptr(t: torch.Tensor | None, dtype=None, cuda=True) -> int | None:
@@ -156,6 +166,14 @@ class Context:
 
     def last_kernel(self) -> str:
         return self.lib.specdec_last_kernel(self.handle).decode()
+
+    def set_phase_stamps(self, stamps: torch.Tensor | None):
+        """specdec_set_phase_stamps of the C ABI: `stamps` is an int64 device tensor [units, STAMP_SLOTS, 2]
+        (or None to switch the timestamps off); needs the diagnostic build of the library."""
+        if stamps is None:
+            self._check(self.lib.specdec_set_phase_stamps(self.handle, None, 0))
+        else:
+            self._check(self.lib.specdec_set_phase_stamps(self.handle, _ptr(stamps, torch.int64), stamps.shape[0]))
 
     def device_status(self, stream=None) -> int:
         """Synchronises the stream; returns the SPECDEC_DATA_* bits (0 = clean) and clears them."""
