@@ -518,9 +518,12 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
-PHASES = [("CTA start -> length known", 0, 1), ("length known -> first row loads issued", 1, 10),
-          ("first loads issued -> first thread's statistics done", 10, 2), ("statistics done -> CTA merged", 2, 3),
-          ("merged -> accept test + draw decision", 3, 4), ("decision -> seen by the CTA", 4, 5),
+PHASES = [("CTA start -> length known", 0, 1), ("length known -> scalars requested", 1, 10),
+          ("scalars requested -> first thread's statistics done", 10, 2), ("statistics done -> CTA merged", 2, 3),
+
+          ("merged -> accept test + draw decision", 3, 4), ("  of which: warp 0 merges the warps' sums", 3, 11),
+          ("  of which: log-probabilities and ratio", 11, 12), ("  of which: flag and optional outputs stored", 12, 13),
+          ("  of which: earlier flags looked up, normalisers", 13, 4), ("decision -> seen by the CTA", 4, 5),
           ("draw: slab sums", 5, 6), ("draw: prefix, slab walk", 6, 7), ("no draw: decision -> arrival", 5, 7),
           ("arrival counted on the row", 7, 8), ("last arriver: ballot + outputs", 8, 9), ("whole unit", 0, 9)]
 
@@ -557,7 +560,7 @@ def run_phases(args, cfg):
     ctx.set_phase_stamps(stamps)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     durs = {name: [] for name, _, _ in PHASES}
-    done_at, start_at, ev_ms, span = [], [], [], []
+    done_at, start_at, ev_ms, span, mhz, skew, wait0 = [], [], [], [], [], [], []
     for i in range(args.steps):
         stamps.zero_()
         e0.record()
@@ -572,18 +575,28 @@ def run_phases(args, cfg):
         start_at.append(np.sort(g[live, 0] - t0) * 1e-3)
         done_at.append(np.sort(g[live, 9] - t0) * 1e-3)
         span.append((g[live, 9].max() - t0) * 1e-3)
+        # durations inside a unit from the SM's cycle counter (the global timer ticks too coarsely for them),
+        # converted with the cycles per nanosecond seen over whole units
+        ghz = float(np.median((c[live, 9] - c[live, 0]) / np.maximum(g[live, 9] - g[live, 0], 1.0)))
+        mhz.append(1e3 * ghz)
         for name, a, b in PHASES:
             ok = live & (c[:, a] > 0) & (c[:, b] > 0)
             if name.startswith("no draw"):
                 ok &= c[:, 6] == 0
-            durs[name].append((g[ok, b] - g[ok, a]) * 1e-3)
+            durs[name].append((c[ok, b] - c[ok, a]) / ghz * 1e-3)
+        wdone = np.where(c[live, 16:32] > 0, c[live, 16:32], np.nan)
+        skew.append((np.nanmax(wdone, 1) - np.nanmin(wdone, 1)) / ghz * 1e-3)
+        wait0.append((c[live, 11] - c[live, 16]) / ghz * 1e-3)
     q = lambda x, p: float(np.percentile(x, p)) if len(x) else float("nan")
     print(f"workload {cfg.name}: B={cfg.B} K={cfg.K} V={cfg.V} {cfg.dtype}, kernel {ctx.last_kernel()}, {args.steps} cold calls; "
-          f"times in us from the device's globaltimer (resolution {np.min(np.diff(np.unique(st[:, :, 0])))} ns)")
+          f"phase durations in us from the SM cycle counters ({np.median(mhz):.0f} MHz), unit start / finish times from the device's global timer")
     print(f"call by CUDA events: mean {1e3 * np.mean(ev_ms):.1f} us; first CTA start -> last unit end: mean {np.mean(span):.1f} us")
     print("| phase | units per call | median | p10 | p90 | max |\n|---|---|---|---|---|---|")
     for name, _, _ in PHASES:
         x = np.concatenate(durs[name])
+        print(f"| {name} | {len(x) // args.steps} | {q(x, 50):.2f} | {q(x, 10):.2f} | {q(x, 90):.2f} | {q(x, 100):.2f} |")
+    for name, x in (("first warp's statistics done -> last warp's", np.concatenate(skew)),
+                    ("warp 0's statistics done -> warps' sums merged by warp 0", np.concatenate(wait0))):
         print(f"| {name} | {len(x) // args.steps} | {q(x, 50):.2f} | {q(x, 10):.2f} | {q(x, 90):.2f} | {q(x, 100):.2f} |")
     sa, da = np.mean(np.stack(start_at), 0), np.mean(np.stack(done_at), 0)
     n = len(sa)

@@ -103,13 +103,14 @@ const char* specdec_last_kernel(const specdec_ctx* ctx);
  * SPECDEC_EUNSUPPORTED for a non-NULL buffer.  After this call every specdec_verify_correct on the
  * context whose B*(K+1) <= units makes each (row, position) unit u = i*B + b write
  * SPECDEC_STAMP_SLOTS pairs {globaltimer in ns, SM cycle counter} at stamps[(u*SLOTS + slot)*2]:
- * slot 0 CTA started, 1 candidate length known, 10 first row loads issued, 2 first thread's share of
+ * slot 0 CTA started, 1 candidate length known, 10 scalar operands requested, 2 first thread's share of
  * the statistics pass done, 3 CTA-wide merge done, 4 accept test and draw decision taken, 5 decision
- * seen by all threads, 6 slab sums of the draw done, 7 draw done, 8 arrival counted on the row,
- * 9 unit finished.  Slots a unit does not reach keep what the caller put there.  stamps = NULL
+ * seen by all threads (11-13 inside the accept test: warps' sums merged, ratio formed, flag stored),
+ * 6 slab sums of the draw done, 7 draw done, 8 arrival counted on the row,
+ * 9 unit finished, 16+w warp w's share of the statistics pass done (w < 16).  Slots a unit does not reach keep what the caller put there.  stamps = NULL
  * switches it off.  The buffer (dev, 16*units*SPECDEC_STAMP_SLOTS bytes) stays the caller's.
  */
-#define SPECDEC_STAMP_SLOTS 16
+#define SPECDEC_STAMP_SLOTS 32
 int specdec_set_phase_stamps(specdec_ctx* ctx, uint64_t* stamps, size_t units);
 
 /*

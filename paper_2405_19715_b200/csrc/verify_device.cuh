@@ -20,9 +20,9 @@ constexpr int FLAG_ACCEPT = 1, FLAG_REJECT = 2, FLAG_BAD = 3;
 __device__ __forceinline__ void stamp(const VerifyParams& P, int unit, int slot) {
 #ifdef SPECDEC_STAMPS
     if (P.stamps) {
-        unsigned long long g;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g));
-        const unsigned long long c = (unsigned long long)clock64();
+        unsigned long long g, c;     // "memory": the reads keep their place between barriers and memory operations
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)::"memory");
+        asm volatile("mov.u64 %0, %%clock64;" : "=l"(c)::"memory");
         unsigned long long* o = P.stamps + ((size_t)unit * SPECDEC_STAMP_SLOTS + slot) * 2;
         o[0] = g;
         o[1] = c;
@@ -308,6 +308,27 @@ __device__ __forceinline__ float ld_early_logit(const __nv_bfloat16* p) {
     return __uint_as_float((uint32_t)v << 16);
 }
 
+// Scalars fetched into shared memory by asynchronous 4-byte copies.  Unlike a load into a register,
+// whose place in the instruction stream the assembler is free to move down to the first use, the
+// copy is in flight from the moment it is issued: a scalar asked for before the streaming pass has
+// landed long before the pass ends.  scalars_wait() by the issuing thread, then a barrier, make them
+// readable by the CTA.
+__device__ __forceinline__ void scalar_fetch(uint32_t* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+                 : "memory");
+}
+__device__ __forceinline__ void scalars_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+// Element e of a row as fp32, fetched as the aligned 4-byte word that holds it (a bf16 element is one
+// half of its word).  The word lies inside the tensor whenever the tensor's base is 4-byte aligned.
+__device__ __forceinline__ void logit_fetch(uint32_t* smem_dst, const float* row, int e) { scalar_fetch(smem_dst, row + e); }
+__device__ __forceinline__ void logit_fetch(uint32_t* smem_dst, const __nv_bfloat16* row, int e) {
+    scalar_fetch(smem_dst, reinterpret_cast<const void*>(reinterpret_cast<uintptr_t>(row + e) & ~(uintptr_t)3));
+}
+__device__ __forceinline__ float logit_fetched(uint32_t w, const float*, int) { return __uint_as_float(w); }
+__device__ __forceinline__ float logit_fetched(uint32_t w, const __nv_bfloat16* row, int e) {
+    return (reinterpret_cast<uintptr_t>(row + e) & 2) ? __uint_as_float(w & 0xffff0000u) : __uint_as_float(w << 16);
+}
+
 // Pass over the two rows of one unit by a CTA of THREADS threads: this thread's share of the
 // softmax statistics (merge with warp_merge / acc_merge).  The draft row is skipped at a bonus
 // position.  VEC: four vectors of each row in flight per thread; the reference is moved from the
@@ -385,6 +406,7 @@ struct UnitShared {
     int need_draw;             // 0 none, 1 residual, 2 target itself
     int token;
     double total;
+    uint32_t pre[4];           // scalars fetched ahead: r_i, the words holding t_y and d_y, the uniform of the draw
 };
 
 struct Unit {
@@ -406,7 +428,7 @@ __device__ __forceinline__ float ratio_from_logs(float lp, float lq) {
 // Flags are plain gpu-scope stores: a flag is self-contained (it carries the call's epoch), and
 // the row's arrival counter orders it for the final ballot.
 __device__ __forceinline__ int unit_accept(const VerifyParams& P, const Unit& u, const Acc& ap, const Acc& aq,
-                                           float t_y, float d_y, int y_ok, float r, int lane) {
+                                           float t_y, float d_y, int y_ok, float r, int lane, int stamp_unit = -1) {
     const int K = P.K;
     const float LN2 = 0.6931471805599453f;
     int state = 0;
@@ -417,6 +439,7 @@ __device__ __forceinline__ int unit_accept(const VerifyParams& P, const Unit& u,
             const float lp = fmaf(t_y, P.c, -ap.rs) - log2f(ap.s);
             const float lq = fmaf(d_y, P.c, -aq.rs) - log2f(aq.s);
             const float ratio = ratio_from_logs(lp, lq);
+            if (stamp_unit >= 0) stamp(P, stamp_unit, 12);
             state = !y_ok ? FLAG_BAD : (r >= ratio ? FLAG_REJECT : FLAG_ACCEPT);   // r == ratio rejects
             if (!y_ok) atomicOr(P.status, SPECDEC_DATA_BAD_TOKEN);
             if (P.ratio) P.ratio[(size_t)u.b * K + u.i] = y_ok ? fminf(1.f, ratio) : -1.f;
@@ -434,6 +457,7 @@ __device__ __forceinline__ int unit_accept(const VerifyParams& P, const Unit& u,
             reinterpret_cast<float4*>(P.stats)[(size_t)u.b * (K + 1) + u.i] = st;
         }
     }
+    if (lane == 0 && stamp_unit >= 0) stamp(P, stamp_unit, 13);
     return __shfl_sync(0xffffffffu, state, 0);
 }
 
@@ -442,8 +466,8 @@ __device__ __forceinline__ int unit_accept(const VerifyParams& P, const Unit& u,
 // needed only if this position can be the first rejection (or is the bonus position); it is
 // skipped when an earlier position of the row is already known to have rejected.
 __device__ __forceinline__ int unit_decide(const VerifyParams& P, const Unit& u, const Acc& ap, const Acc& aq,
-                                           float t_y, float d_y, int y_ok, float r, int lane) {
-    const int state = unit_accept(P, u, ap, aq, t_y, d_y, y_ok, r, lane);
+                                           float t_y, float d_y, int y_ok, float r, int lane, int stamp_unit = -1) {
+    const int state = unit_accept(P, u, ap, aq, t_y, d_y, y_ok, r, lane, stamp_unit);
     if (!u.bonus && state != FLAG_REJECT) return 0;      // accepted (or bad token): never draws
     bool known = false;
     for (int j0 = 0; j0 < u.i; j0 += 32) {

@@ -24,16 +24,14 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
     // 4 accept test and draw decision, 5 decision seen by the CTA, 6 slab sums, 7 draw done, 8 arrival counted, 9 end
     if (tid == 0) stamp(P, unit, 0);
 
-    // Everything the accept test needs besides the sums.  The length, the uniform and the drafted
-    // token are requested together (their addresses do not depend on the length), the two logits of
-    // the drafted token right behind the first row loads: one round trip instead of three in a row.
+    // Everything the accept test needs besides the sums.  The length and the drafted token are requested
+    // together (their addresses do not depend on the length); once they are known, thread 0 starts
+    // asynchronous copies of the uniform of the accept test, of the two logits of the drafted token and
+    // of the uniform of the draw into shared memory, and the streaming pass begins: the scalars land
+    // while it runs instead of costing dependent round trips after it.
     u.L = P.lens ? ld_early_s32(P.lens + u.b) : P.K;
-    float r = 0.f;
     int y = 0;
-    if (tid == 0 && u.i < P.K) {
-        r = ld_early_f32(P.uniforms + (size_t)u.b * (P.K + 1) + u.i);
-        y = ld_early_s32(P.tokens + (size_t)u.b * P.K + u.i);
-    }
+    if (tid == 0 && u.i < P.K) y = ld_early_s32(P.tokens + (size_t)u.b * P.K + u.i);
     if (u.L < 0 || u.L > P.K) {                  // bad length: the row reports -1, nothing is read
         if (u.i == 0 && tid == 0) {
             atomicOr(P.status, SPECDEC_DATA_BAD_LENGTH);
@@ -52,19 +50,22 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
     const T* drow = u.bonus ? trow : static_cast<const T*>(P.draft) + ((size_t)u.b * P.K + u.i) * V;
 
     int y_ok = 1;
-    float t_y = 0.f, d_y = 0.f;
-    auto gather_y = [&]() {
-        if (tid == 0) stamp(P, unit, 10);        // first round of row loads issued
-        if (tid == 0 && !u.bonus) {
+    if (tid == 0) {
+        const float* ur = P.uniforms + (size_t)u.b * (P.K + 1);
+        scalar_fetch(&sh.pre[3], ur + P.K);
+        if (!u.bonus) {
+            scalar_fetch(&sh.pre[0], ur + u.i);
             y_ok = (y >= 0 && y < P.V);
-            if (y_ok) { t_y = ld_early_logit(trow + y); d_y = ld_early_logit(drow + y); }
+            if (y_ok) { logit_fetch(&sh.pre[1], trow, y); logit_fetch(&sh.pre[2], drow, y); }
         }
-    };
+        stamp(P, unit, 10);                      // scalars requested
+    }
 
     // ---- pass 1: softmax statistics of both rows
     Acc ap = acc_init(), aq = acc_init();
-    unit_stats<T, VEC, THREADS>(trow, drow, P.V, P.c, u.bonus, tid, ap, aq, gather_y);
-    if (tid == 0) stamp(P, unit, 2);
+    unit_stats<T, VEC, THREADS>(trow, drow, P.V, P.c, u.bonus, tid, ap, aq);
+    if (tid == 0) { stamp(P, unit, 2); scalars_wait(); }
+    if (lane == 0 && warp < 16) stamp(P, unit, 16 + warp);
     warp_merge2(ap, aq);
     if (lane == 0) { sh.wp[warp] = ap; sh.wq[warp] = aq; }
     __syncthreads();
@@ -73,7 +74,10 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
         constexpr int NW = THREADS / 32;
         Acc a = lane < NW ? sh.wp[lane] : acc_init(), b = lane < NW ? sh.wq[lane] : acc_init();
         warp_merge2(a, b);
-        const int mode = unit_decide(P, u, a, b, t_y, d_y, y_ok, r, lane);
+        if (lane == 0) stamp(P, unit, 11);
+        const float r = __uint_as_float(sh.pre[0]);
+        const float t_y = logit_fetched(sh.pre[1], trow, y), d_y = logit_fetched(sh.pre[2], drow, y);
+        const int mode = unit_decide(P, u, a, b, t_y, d_y, y_ok, r, lane, unit);
         if (lane == 0) {
             sh.np = make_norm(a);
             sh.nq = u.bonus ? sh.np : make_norm(b);
@@ -87,7 +91,7 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
     // ---- pass 2 (only where this position may supply y'): weights, prefix, inverse CDF
     const int mode = sh.need_draw;
     if (mode) {
-        const float u01 = P.uniforms[(size_t)u.b * (P.K + 1) + P.K];
+        const float u01 = __uint_as_float(sh.pre[3]);
         unit_draw<T, VEC>(P, trow, drow, mode, u01, sh, slab_sum, tid, THREADS, 0, -1.0, unit);
         if (mode == 1 && !(sh.total > 1e-30)) {   // p == q to rounding: draw from p itself
             const double keep = sh.total;

@@ -23,7 +23,7 @@ EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_d
            "specdec_shard_stats", "specdec_shard_accept", "specdec_shard_draw"]
 SHARD_STATS_WIDTH, SHARD_MAX_RANKS = 8, 64
 STATIC_MAX_UNITS, STATIC_MAX_V = 16384, 262144
-STAMP_SLOTS = 16
+STAMP_SLOTS = 32
 
 
 class SpecdecError(RuntimeError):
