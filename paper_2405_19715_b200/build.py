@@ -11,7 +11,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libspecdec.so"
-SOURCES = ["api.cu", "verify.cu", "verify_stream.cu", "stop.cu", "head.cu", "verify_static.cu", "greedy.cu", "topk.cu", "verify_shard.cu", "verify_cluster.cu"]
+SOURCES = ["api.cu", "verify.cu", "verify_stream.cu", "stop.cu", "head.cu", "verify_static.cu", "greedy.cu", "topk.cu", "verify_shard.cu", "verify_cluster.cu", "verify_split.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--expt-relaxed-constexpr"]
 
@@ -59,7 +59,7 @@ def _compile(LIB: Path, obj_dir: Path, defines: list, verbose: bool) -> Path:
     if failed:
         raise RuntimeError("nvcc failed building libspecdec")
     tmp = LIB.with_suffix(".so.tmp%d" % os.getpid())
-    cmd = [nvcc, "-shared", "-o", str(tmp), *[str(obj_dir / (s + ".o")) for s in SOURCES], "-lcudart"]
+    cmd = [nvcc, "-shared", "-Wno-deprecated-gpu-targets", "-o", str(tmp), *[str(obj_dir / (s + ".o")) for s in SOURCES], "-lcudart"]
     subprocess.run(cmd, check=True)
     os.replace(tmp, LIB)
     return LIB

@@ -12,53 +12,13 @@
 //
 // Every CTA of a cluster executes the same sequence of cluster barriers; early exits depend on the
 // unit only, so they are taken by the whole cluster.
-#include "verify_device.cuh"
+#include "verify_cluster.cuh"
 
 namespace {
 
 using namespace sd;
 
 constexpr int CL_THREADS = 512;
-constexpr int CL_MAX = 8;                          // portable cluster size limit
-
-struct ClusterShared {
-    Acc part_p, part_q;                            // this CTA's slice statistics
-    double total;                                  // this CTA's slice mass
-    double W;                                      // mass of the whole row (local copy)
-    int mode;                                      // CTA 0: 0 no draw, 1 residual, 2 target itself
-    int mode_l;                                    // local copy of CTA 0's decision
-};
-
-__device__ __forceinline__ uint32_t cl_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cl_sync() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Address of `p` (own shared memory) as seen in CTA `rank` of the cluster.
-__device__ __forceinline__ uint32_t cl_map(const void* p, uint32_t rank) {
-    uint32_t a = (uint32_t)__cvta_generic_to_shared(p), r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ float cl_ld_f32(uint32_t a) {
-    float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ double cl_ld_f64(uint32_t a) {
-    double v;
-    asm volatile("ld.shared::cluster.f64 %0, [%1];" : "=d"(v) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ int cl_ld_s32(uint32_t a) {
-    int v;
-    asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
-    return v;
-}
 
 template <typename T, bool VEC>
 __global__ void __launch_bounds__(CL_THREADS) verify_cluster_kernel(const VerifyParams P, int C, int slice_len) {
@@ -73,15 +33,12 @@ __global__ void __launch_bounds__(CL_THREADS) verify_cluster_kernel(const Verify
     u.i = unit / P.B;
     u.b = unit - u.i * P.B;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // length, uniform and drafted token are requested together; the drafted token's two logits
-    // right behind the first row loads
+    // length and drafted token are requested together; once they are known CTA 0 starts asynchronous
+    // copies of the accept test's uniform and of the drafted token's two logits into shared memory,
+    // every CTA one of the uniform of the draw
     u.L = P.lens ? ld_early_s32(P.lens + u.b) : P.K;
-    float r = 0.f;
     int y = 0;
-    if (rank == 0 && tid == 0 && u.i < P.K) {
-        r = ld_early_f32(P.uniforms + (size_t)u.b * (P.K + 1) + u.i);
-        y = ld_early_s32(P.tokens + (size_t)u.b * P.K + u.i);
-    }
+    if (rank == 0 && tid == 0 && u.i < P.K) y = ld_early_s32(P.tokens + (size_t)u.b * P.K + u.i);
     if (u.L < 0 || u.L > P.K) {                    // bad length: the row reports -1, nothing is read
         if (u.i == 0 && rank == 0 && tid == 0) {
             atomicOr(P.status, SPECDEC_DATA_BAD_LENGTH);
@@ -106,17 +63,20 @@ __global__ void __launch_bounds__(CL_THREADS) verify_cluster_kernel(const Verify
     Ps.V = len;
 
     int y_ok = 1;
-    float t_y = 0.f, d_y = 0.f;
-    auto gather_y = [&]() {
-        if (rank == 0 && tid == 0 && !u.bonus) {
+    if (tid == 0) {
+        const float* ur = P.uniforms + (size_t)u.b * (P.K + 1);
+        scalar_fetch(&sh.pre[3], ur + P.K);
+        if (rank == 0 && !u.bonus) {
+            scalar_fetch(&sh.pre[0], ur + u.i);
             y_ok = (y >= 0 && y < P.V);
-            if (y_ok) { t_y = ld_early_logit(trow + y); d_y = ld_early_logit(drow + y); }
+            if (y_ok) { logit_fetch(&sh.pre[1], trow, y); logit_fetch(&sh.pre[2], drow, y); }
         }
-    };
+    }
 
     // ---- statistics of the slice
     Acc ap = acc_init(), aq = acc_init();
-    unit_stats<T, VEC, CL_THREADS>(ts, ds, len, P.c, u.bonus, tid, ap, aq, gather_y);
+    unit_stats<T, VEC, CL_THREADS>(ts, ds, len, P.c, u.bonus, tid, ap, aq);
+    if (tid == 0) scalars_wait();
     warp_merge2(ap, aq);
     if (lane == 0) { sh.wp[warp] = ap; sh.wq[warp] = aq; }
     __syncthreads();
@@ -148,6 +108,8 @@ __global__ void __launch_bounds__(CL_THREADS) verify_cluster_kernel(const Verify
             gq = acc_merge(gq, b);
         }
         if (rank == 0) {
+            const float r = __uint_as_float(sh.pre[0]);
+            const float t_y = logit_fetched(sh.pre[1], trow, y), d_y = logit_fetched(sh.pre[2], drow, y);
             const int mode = unit_decide(P, u, gp, gq, t_y, d_y, y_ok, r, lane);
             if (lane == 0) cs.mode = mode;
         }
@@ -167,57 +129,11 @@ __global__ void __launch_bounds__(CL_THREADS) verify_cluster_kernel(const Verify
     }
 
     // ---- the draw: slice masses, the slice that holds u * W, a walk inside it
-    const int nvec = (len + N - 1) / N, nslab = (nvec + 31) / 32;
-    double W_report = 0.0;
-    for (int pass = 0; pass < 2; ++pass) {
-        unit_slabs<T, VEC>(Ps, ts, ds, mode, sh.np, sh.nq, slab_sum, tid, CL_THREADS);
-        __syncthreads();
-        if (warp == 0) {
-            const double tot = slab_total(slab_sum, nslab, lane);
-            if (lane == 0) cs.total = tot;
-        }
-        cl_sync();                                 // every slice's mass is in place
-        if (warp == 0) {
-            const double m = lane < C ? cl_ld_f64(cl_map(&cs.total, lane)) : 0.0;
-            double W = 0.0;
-            for (int k = 0; k < C; ++k) W += __shfl_sync(0xffffffffu, m, k);
-            if (lane == 0) cs.W = W;
-        }
-        __syncthreads();
-        if (pass == 0) W_report = cs.W;
-        if (pass == 0 && mode == 1 && !(cs.W > 1e-30)) {   // p == q to rounding: draw from p itself (cluster-uniform)
-            mode = 2;
-            cl_sync();                             // all masses have been read before they are overwritten
-            continue;
-        }
-        break;
-    }
-    if (warp == 0) {
-        const double m = lane < C ? cl_ld_f64(cl_map(&cs.total, lane)) : 0.0;
-        const float u01 = P.uniforms[(size_t)u.b * (P.K + 1) + P.K];
-        const double thr = (double)u01 * cs.W;
-        int owner = -1, lastpos = -1;
-        double before = 0.0, run = 0.0;
-        for (int k = 0; k < C; ++k) {
-            const double mk = __shfl_sync(0xffffffffu, m, k);
-            if (mk > 0.0) lastpos = k;
-            if (owner < 0 && run + mk > thr) { owner = k; before = run; }
-            run += mk;
-        }
-        if (owner < 0) {                           // rounding left nothing above u * W: the last slice with mass
-            owner = lastpos < 0 ? 0 : lastpos;
-            before = 0.0;
-            for (int k = 0; k < owner; ++k) before += __shfl_sync(0xffffffffu, m, k);
-        }
-        if (owner == (int)rank) {
-            double total;
-            const double tau = thr - before;
-            const int tok = draw_select<T, VEC>(Ps, ts, ds, mode, u01, sh.np, sh.nq, slab_sum, lane, &total,
-                                                tau > 0.0 ? tau : 0.0);
-            unit_finish(P, u, 1, start + tok, (float)W_report, lane);
-        }
-    }
-    cl_sync();                                     // nobody leaves while its mass may still be read
+    int tok = -1;
+    double W = 0.0;
+    const float u01 = __uint_as_float(sh.pre[3]);
+    if (cluster_draw<T, VEC, CL_THREADS>(Ps, ts, ds, start, len, mode, u01, sh.np, sh.nq, C, rank, cs, slab_sum, &tok, &W))
+        unit_finish(P, u, 1, tok, (float)W, lane);
 }
 
 template <typename T>
@@ -225,11 +141,8 @@ cudaError_t launch_t(const VerifyParams& p, int C, cudaStream_t s) {
     constexpr int N = Elem<T>::EPV;
     const bool vec = (p.V % N == 0) && (reinterpret_cast<uintptr_t>(p.target) % 16 == 0) &&
                      (reinterpret_cast<uintptr_t>(p.draft) % 16 == 0);
-    // slices of whole slabs (32 vectors), so that a slice is as well aligned as the row
-    const int nvec = (p.V + N - 1) / N;
-    const int slabs = (nvec + 31) / 32, slab_per = (slabs + C - 1) / C;
-    const int slice_len = slab_per * 32 * N;
-    const size_t smem = (size_t)slab_per * sizeof(float);
+    const int slice_len = cluster_slice_len<T>(p.V, C);
+    const size_t smem = (size_t)(slice_len / (32 * N)) * sizeof(float);
     auto kern = vec ? verify_cluster_kernel<T, true> : verify_cluster_kernel<T, false>;
     if (smem > 40 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -495,20 +495,16 @@ __device__ __forceinline__ float vec_weights(const float (&xt)[N], const float (
 }
 
 // Second half of a draw, run by one full warp once every slab sum is in `slab_sum`: fp64 prefix
-// over the slabs, the slab that holds u * total, then a walk inside that slab (its vectors are
-// re-read from global memory).  Returns the token; *total_out receives the total mass.
-template <typename T, bool VEC>
-__device__ __forceinline__ int draw_select(const VerifyParams& P, const T* __restrict__ trow,
-                                           const T* __restrict__ drow, int mode, float u01, const Norm np,
-                                           const Norm nq, const float* __restrict__ slab_sum, int lane,
-                                           double* total_out, double tau_abs = -1.0) {
-    constexpr int N = Elem<T>::EPV;
-    const int V = P.V;
-    const int nvec = (V + N - 1) / N;
-    const int nslab = (nvec + 31) / 32;
-    float xt[N], xd[N], w[N];
-#pragma unroll
-    for (int k = 0; k < N; ++k) xd[k] = 0.f;
+// over the slabs and the slab that holds the mass to walk to (draw_find), then a walk inside that
+// slab over one vector of weights per lane (draw_walk).
+struct SlabPick {
+    int slab;                  // the slab that holds tau
+    double base;               // mass of the slabs before it
+    double tau;                // the mass to walk to
+    double total;              // mass of all slabs
+};
+__device__ __forceinline__ SlabPick draw_find(const float* __restrict__ slab_sum, int nslab, float u01, int lane,
+                                              double tau_abs = -1.0) {
     // fp64 prefix over slabs: each lane owns a contiguous run of slabs
     const int per = (nslab + 31) / 32;
     const int s0 = min(lane * per, nslab), s1 = min(s0 + per, nslab);
@@ -520,24 +516,24 @@ __device__ __forceinline__ int draw_select(const VerifyParams& P, const T* __res
         const double up = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += up;
     }
-    const double total = __shfl_sync(0xffffffffu, incl, 31);
-    // the mass to walk to: u * total, unless the caller fixed it (a draw that spans several calls' rows)
-    const double tau = tau_abs >= 0.0 ? tau_abs : (double)u01 * total;
+    SlabPick pk;
+    pk.total = __shfl_sync(0xffffffffu, incl, 31);
+    // the mass to walk to: u * total, unless the caller fixed it (a draw that spans several CTAs' slices)
+    pk.tau = tau_abs >= 0.0 ? tau_abs : (double)u01 * pk.total;
     // first slab whose inclusive prefix exceeds tau
     double run = incl - mine;
     int found = -1;
     double base = 0.0;
     for (int s = s0; s < s1; ++s) {
         const double nxt = run + (double)slab_sum[s];
-        if (found < 0 && nxt > tau) { found = s; base = run; }
+        if (found < 0 && nxt > pk.tau) { found = s; base = run; }
         run = nxt;
     }
     const unsigned m = __ballot_sync(0xffffffffu, found >= 0);
-    int slab;
     if (m) {
         const int src = __ffs(m) - 1;
-        slab = __shfl_sync(0xffffffffu, found, src);
-        base = __shfl_sync(0xffffffffu, base, src);
+        pk.slab = __shfl_sync(0xffffffffu, found, src);
+        pk.base = __shfl_sync(0xffffffffu, base, src);
     } else {
         // rounding left nothing above tau: take the last slab with positive mass
         int lastpos = -1;
@@ -549,20 +545,18 @@ __device__ __forceinline__ int draw_select(const VerifyParams& P, const T* __res
         }
         const unsigned pm = __ballot_sync(0xffffffffu, lastpos >= 0);
         const int src = pm ? 31 - __clz(pm) : 0;
-        slab = __shfl_sync(0xffffffffu, lastpos, src);
-        base = __shfl_sync(0xffffffffu, lb, src);
-        if (slab < 0) { slab = 0; base = 0.0; }
+        pk.slab = __shfl_sync(0xffffffffu, lastpos, src);
+        pk.base = __shfl_sync(0xffffffffu, lb, src);
+        if (pk.slab < 0) { pk.slab = 0; pk.base = 0.0; }
     }
-    // walk inside the slab
-    const int j = slab * 32 + lane;
-    float ls = 0.f;
-#pragma unroll
-    for (int k = 0; k < N; ++k) w[k] = 0.f;
-    if (j < nvec) {
-        load_vec<T, VEC>(trow, j, V, xt);
-        if (mode == 1) load_vec<T, VEC>(drow, j, V, xd);
-        ls = vec_weights<N>(xt, xd, P.c, np, nq, mode, w);
-    }
+    return pk;
+}
+
+// Walk inside slab pk.slab: lane l holds the N weights w of vector pk.slab * 32 + l (zeros past the row's
+// end) and their fp32 sum ls.  Returns the token in every lane.
+template <int N>
+__device__ __forceinline__ int draw_walk(const SlabPick& pk, const float (&w)[N], float ls, int V, int lane) {
+    const int j = pk.slab * 32 + lane;
     float li = ls;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -571,25 +565,50 @@ __device__ __forceinline__ int draw_select(const VerifyParams& P, const T* __res
     }
     float lex = __shfl_up_sync(0xffffffffu, li, 1);
     if (lane == 0) lex = 0.f;
-    const unsigned hm = __ballot_sync(0xffffffffu, base + (double)li > tau);
+    const unsigned hm = __ballot_sync(0xffffffffu, pk.base + (double)li > pk.tau);
     const unsigned pm = __ballot_sync(0xffffffffu, ls > 0.f);
     const int sel = hm ? __ffs(hm) - 1 : (pm ? 31 - __clz(pm) : -1);
-    int tok = min(slab * 32 * N, V - 1);
+    int tok = min(pk.slab * 32 * N, V - 1);
     if (sel >= 0 && lane == sel) {
-        double acc = base + (double)lex;
+        double acc = pk.base + (double)lex;
         int pick = -1, lastp = 0;
 #pragma unroll
         for (int k = 0; k < N; ++k) {
             acc += (double)w[k];
             if (w[k] > 0.f) lastp = k;
-            if (pick < 0 && acc > tau) pick = k;
+            if (pick < 0 && acc > pk.tau) pick = k;
         }
         if (pick < 0) pick = lastp;
         tok = min(j * N + pick, V - 1);
     }
     if (sel >= 0) tok = __shfl_sync(0xffffffffu, tok, sel);
-    *total_out = total;
     return tok;
+}
+
+// draw_find, then the chosen slab's vectors re-read from global memory, then draw_walk.  Returns the
+// token; *total_out receives the total mass.
+template <typename T, bool VEC>
+__device__ __forceinline__ int draw_select(const VerifyParams& P, const T* __restrict__ trow,
+                                           const T* __restrict__ drow, int mode, float u01, const Norm np,
+                                           const Norm nq, const float* __restrict__ slab_sum, int lane,
+                                           double* total_out, double tau_abs = -1.0) {
+    constexpr int N = Elem<T>::EPV;
+    const int V = P.V;
+    const int nvec = (V + N - 1) / N;
+    const int nslab = (nvec + 31) / 32;
+    const SlabPick pk = draw_find(slab_sum, nslab, u01, lane, tau_abs);
+    float xt[N], xd[N], w[N];
+#pragma unroll
+    for (int k = 0; k < N; ++k) { xd[k] = 0.f; w[k] = 0.f; }
+    const int j = pk.slab * 32 + lane;
+    float ls = 0.f;
+    if (j < nvec) {
+        load_vec<T, VEC>(trow, j, V, xt);
+        if (mode == 1) load_vec<T, VEC>(drow, j, V, xd);
+        ls = vec_weights<N>(xt, xd, P.c, np, nq, mode, w);
+    }
+    *total_out = pk.total;
+    return draw_walk<N>(pk, w, ls, V, lane);
 }
 
 // First half of a block-wide draw: the fp32 sum of the weights of every slab of the rows (read from
