@@ -690,7 +690,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=sorted(wl.CONFIGS))
-    ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 one CTA per unit, 2 two-launch TMA pipeline, 3 fused TMA pipeline, 4 cluster per unit, 5 statistics launch + draw launch")
+    ap.add_argument("--kernel", type=int, default=0, help="0 auto, 1 one CTA per unit, 2 two-launch TMA pipeline, 3 fused TMA pipeline, 4 cluster per unit")
     ap.add_argument("--top-k", type=int, default=0,
                     help="verify under top-k sampling (the paper's runs use 50); 0 = whole vocabulary, the headline workload")
     ap.add_argument("--vocab-shards", action="store_true",

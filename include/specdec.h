@@ -71,9 +71,6 @@ typedef enum {
                                     a slice of the vocabulary, combined through distributed shared
                                     memory; picked automatically while the units fit the SMs twice   */
 
-#define SPECDEC_VERIFY_SPLIT   5u /* two launches: statistics and accept tests with one narrow CTA per (row,
-                                    position), then one cluster per row for the first rejection and the draw */
-
 /*
  * Create a context on `device` able to serve calls with B <= max_B and K <= max_K.
  * Allocates the scratch used by verify/correct (per-(row,position) flags and draws,

@@ -11,7 +11,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libspecdec.so"
-SOURCES = ["api.cu", "verify.cu", "verify_stream.cu", "stop.cu", "head.cu", "verify_static.cu", "greedy.cu", "topk.cu", "verify_shard.cu", "verify_cluster.cu", "verify_split.cu"]
+SOURCES = ["api.cu", "verify.cu", "verify_stream.cu", "stop.cu", "head.cu", "verify_static.cu", "greedy.cu", "topk.cu", "verify_shard.cu", "verify_cluster.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--expt-relaxed-constexpr"]
 

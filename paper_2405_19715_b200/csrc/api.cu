@@ -40,7 +40,7 @@ int check_verify_args(specdec_ctx* ctx, const void* target, const void* draft, i
     if (dtype != SPECDEC_F32 && dtype != SPECDEC_BF16) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown dtype %d", dtype);
     if (B < 1 || K < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "verify_correct: B, K, V must be >= 1 (got %d, %d, %d)", B, K, V);
     if (!(T > 0.f) || !std::isfinite(T)) return fail(ctx, SPECDEC_EINVAL, "verify_correct: temperature must be positive and finite");
-    if (flags > SPECDEC_VERIFY_SPLIT) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown flags %u", flags);
+    if (flags > SPECDEC_VERIFY_CLUSTER) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown flags %u", flags);
     if (B > ctx->max_B || K > ctx->max_K)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: B=%d K=%d exceed the context (max_B=%d max_K=%d)", B, K, ctx->max_B, ctx->max_K);
     if (V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: V=%d above 2^22", V);
@@ -83,9 +83,6 @@ int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_
     if (e == cudaSuccess) e = cudaMemset(ctx->task_ctl, 0, 8 * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->task_ready, (size_t)max_B * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->task_ready, 0, (size_t)max_B * sizeof(int32_t));
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->partials, ((size_t)max_B * (2 * max_K + 1) + 4 * (size_t)ctx->sm_count) * sizeof(float2));
-    if (e == cudaSuccess) e = cudaMalloc(&ctx->unit_arrive, ndraw * sizeof(int32_t));
-    if (e == cudaSuccess) e = cudaMemset(ctx->unit_arrive, 0, ndraw * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->flags, 0, nflag * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->arrive, 0, (size_t)max_B * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMemset(ctx->status, 0, sizeof(uint32_t));
@@ -117,8 +114,6 @@ int specdec_destroy(specdec_ctx* ctx) {
     cudaFree(ctx->tasks);
     cudaFree(ctx->task_ctl);
     cudaFree(ctx->task_ready);
-    cudaFree(ctx->partials);
-    cudaFree(ctx->unit_arrive);
     cudaFree(ctx->stage);
     cudaFree(ctx->act[0]);
     cudaFree(ctx->act[1]);
@@ -201,8 +196,6 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
     p.tasks = ctx->tasks;
     p.task_ctl = ctx->task_ctl;
     p.task_ready = ctx->task_ready;
-    p.partials = ctx->partials;
-    p.unit_arrive = ctx->unit_arrive;
     p.epoch = ctx->epoch;
     if (ctx->stamps && (size_t)B * (K + 1) <= ctx->stamps_units) p.stamps = ctx->stamps;
 
@@ -215,20 +208,17 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
         kind = verify_cluster_size(p, dtype, ctx->sm_count) > 1 ? SPECDEC_VERIFY_CLUSTER : SPECDEC_VERIFY_DIRECT;
     }
     if (kind == SPECDEC_VERIFY_FUSED && K > 63) kind = SPECDEC_VERIFY_STREAM;     // row records hold n in 6 bits
-    if (kind == SPECDEC_VERIFY_SPLIT && !verify_split_supported(p, dtype)) kind = SPECDEC_VERIFY_DIRECT;
     if ((kind == SPECDEC_VERIFY_STREAM || kind == SPECDEC_VERIFY_FUSED) && !stream_ok)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: streaming kernels need 16-byte aligned rows (V=%d)", V);
     int n_launch = 0;
     const int csize = kind == SPECDEC_VERIFY_CLUSTER ? verify_cluster_size(p, dtype, ctx->sm_count) : 1;
     cudaError_t e = kind == SPECDEC_VERIFY_CLUSTER  ? launch_verify_cluster(p, dtype, csize > 1 ? csize : 2, s, &n_launch)
-                    : kind == SPECDEC_VERIFY_SPLIT  ? launch_verify_split(p, dtype, ctx->sm_count, s, &n_launch)
                     : kind == SPECDEC_VERIFY_FUSED  ? launch_verify_fused(p, dtype, ctx->sm_count, s, &n_launch)
                     : kind == SPECDEC_VERIFY_STREAM ? launch_verify_stream(p, dtype, ctx->sm_count, s, &n_launch)
                                                     : launch_verify_direct(p, dtype, s, &n_launch);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "verify_correct launch");
     ctx->launches += n_launch;
     ctx->last_kernel = kind == SPECDEC_VERIFY_CLUSTER  ? "verify_cluster_kernel"
-                       : kind == SPECDEC_VERIFY_SPLIT  ? "verify_split_stats_kernel"
                        : kind == SPECDEC_VERIFY_FUSED  ? "verify_fused_kernel"
                        : kind == SPECDEC_VERIFY_STREAM ? "verify_stream_stats_kernel"
                                                        : "verify_direct_kernel";

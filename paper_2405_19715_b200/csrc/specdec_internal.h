@@ -20,8 +20,6 @@ struct specdec_ctx {
     int2* tasks = nullptr;        // [max_B]              rows whose y' is still to be drawn: {b, n}
     int32_t* task_ctl = nullptr;  // [8]                  two-launch path: {tasks, finished CTAs}; fused path: {-, -, -, head, finished}; [5]: CTAs done in the few-row head block
     int32_t* task_ready = nullptr;// [max_B]              fused path: record {epoch:24, mode:2, n:6} of each resolved row
-    float2* partials = nullptr;   // [max_B * (2 max_K + 1) + 4 * sm_count]  two-launch path: {reference, sum} of every CTA's share of a logit row
-    int32_t* unit_arrive = nullptr;// [max_B * (max_K+1)]  two-launch path: chunks of a unit that have been summed
     uint32_t epoch = 0;
     uint64_t launches = 0;
     const char* last_kernel = "none";   // name of the kernel the last verify/correct call launched
@@ -58,8 +56,6 @@ struct VerifyParams {
     int2* tasks;
     int32_t* task_ctl;
     int32_t* task_ready;
-    float2* partials;
-    int32_t* unit_arrive;
     uint32_t epoch;
     unsigned long long* stamps = nullptr;   // phase timestamps, SPECDEC_STAMP_SLOTS {globaltimer ns, SM clock} pairs per unit (diagnostic builds)
 };
@@ -75,9 +71,6 @@ cudaError_t launch_verify_stream(const VerifyParams& p, specdec_dtype dtype, int
                                  int* n_launch);
 cudaError_t launch_verify_fused(const VerifyParams& p, specdec_dtype dtype, int sm_count, cudaStream_t s,
                                 int* n_launch);
-cudaError_t launch_verify_split(const VerifyParams& p, specdec_dtype dtype, int sm_count, cudaStream_t s,
-                                int* n_launch);
-bool verify_split_supported(const VerifyParams& p, specdec_dtype dtype);
 bool verify_stream_supported(const VerifyParams& p, specdec_dtype dtype);
 cudaError_t launch_greedy(const VerifyParams& p, specdec_dtype dtype, int32_t* argmax_out, cudaStream_t s);
 cudaError_t launch_stop(const float* accept_prob, const int32_t* lens, float h, int B, int K,

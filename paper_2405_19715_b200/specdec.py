@@ -14,7 +14,7 @@ from . import build as _build
 
 F32, BF16 = 0, 1
 OK, EINVAL, EUNSUPPORTED, ECUDA, EDATA = 0, 1, 2, 3, 4
-VERIFY_AUTO, VERIFY_DIRECT, VERIFY_STREAM, VERIFY_FUSED, VERIFY_CLUSTER, VERIFY_SPLIT = 0, 1, 2, 3, 4, 5
+VERIFY_AUTO, VERIFY_DIRECT, VERIFY_STREAM, VERIFY_FUSED, VERIFY_CLUSTER = 0, 1, 2, 3, 4
 DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT, DATA_TOPK_TIES = 1, 2, 4, 8
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",

@@ -9,8 +9,8 @@ from paper_2405_19715_b200 import specdec, workloads as wl  # noqa: E402
 from tests import parity  # noqa: E402
 from oracle.specdec_oracle import stop_rule as orc_stop  # noqa: E402
 
-KERNELS = [specdec.VERIFY_DIRECT, specdec.VERIFY_STREAM, specdec.VERIFY_FUSED, specdec.VERIFY_CLUSTER, specdec.VERIFY_SPLIT]
-KERNEL_IDS = ["direct", "stream", "fused", "cluster", "split"]
+KERNELS = [specdec.VERIFY_DIRECT, specdec.VERIFY_STREAM, specdec.VERIFY_FUSED, specdec.VERIFY_CLUSTER]
+KERNEL_IDS = ["direct", "stream", "fused", "cluster"]
 
 
 @pytest.fixture(scope="module")
