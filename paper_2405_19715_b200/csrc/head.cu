@@ -12,7 +12,9 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdio>
+#include <cstring>
 
 #include "specdec_internal.h"
 
@@ -26,7 +28,7 @@ constexpr int HEAD_THREADS = (2 + EPI_WARPS) * 32;   // warp 0 TMA, warp 1 MMA +
 constexpr uint32_t WAIT_POLLS = 1u << 24;
 
 template <int BN> struct Cfg {
-    static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr int STAGES = BN == 256 ? 4 : 6;
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
@@ -268,6 +270,257 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)(2 * BN)) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The block for 17 to 256 rows (the online use of Eq. 3 for tens to hundreds of concurrent sequences):
+// the GEMM is a stream of the weights against a handful of rows, so the WEIGHTS are the M-side operand.
+// A tile is Z^T[128 output features, N rows of X] = W[128, k] * X^T[k, N]: one tcgen05.mma takes 128
+// weight rows whatever the number of rows of X (N = M rounded up to 16); the accumulator holds one
+// output feature per tensor-memory lane and one row of X per column.  To put the weight stream on as
+// many SMs as the memory system needs, the reduction dimension is split over the KS CTAs of a
+// thread-block cluster: each CTA accumulates its k-slice, then sends the lane quarters of its
+// accumulator to the CTAs that own them (stores into the owners' shared memory), and after a cluster
+// barrier each CTA adds the KS contributions to its 128 / KS features and runs the epilogue for them
+// (bias, SiLU, residual, bf16 store, or the w_out dot of the last block, whose last CTA also adds the
+// dots and applies the sigmoid).  The kernel is launched programmatically dependent on the stream's
+// previous kernel -- the previous block -- and asks for its first ring-full of weight tiles before
+// that kernel has completed; only the rows of X wait for it.
+constexpr int SW_THREADS = 6 * 32;       // warp 0 TMA, warp 1 MMA + tensor-memory owner, warps 2-5 epilogue
+constexpr int SW_UR = 8;                 // rows an epilogue warp works on together
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t local_addr, uint32_t rank, float v) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+
+// Phase timestamps of one CTA (diagnostic builds only): [last block ? 1 : 0][warp][slot], global timer in ns.
+#ifdef SPECDEC_STAMPS
+__device__ long long head_stamps[2 * 6 * 16];
+#define HEAD_STAMP(slot)                                                                         \
+    do {                                                                                         \
+        if (blockIdx.x == 5 && lane == 0) {                                                      \
+            long long t_;                                                                        \
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                               \
+            head_stamps[(P.partial ? 96 : 0) + warp * 16 + (slot)] = t_;                         \
+        }                                                                                        \
+    } while (0)
+#else
+#define HEAD_STAMP(slot) do {} while (0)
+#endif
+
+template <int KS>
+__global__ void __launch_bounds__(SW_THREADS, 1)
+head_swap_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW, const BlockParams P,
+                 int Npad, int stages, int tmem_cols) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* aligned = smem_raw + (base - smem_u32(smem_raw));
+    const int a_bytes = BM * BK * 2, stage_bytes = a_bytes + Npad * BK * 2;
+    const int ring_bytes = max(stages * stage_bytes, 512 * Npad);         // the ring is reused to receive the partial sums
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(aligned + ring_bytes);
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * stages, tfull = empty0 + 8 * stages;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * stages + 2);
+    float* recv = reinterpret_cast<float*>(aligned);                      // [KS][4 / KS][Npad][32]
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    HEAD_STAMP(0);
+    const int rank = (int)cluster_rank();
+    const int n0 = (blockIdx.x / KS) * BM;                                // first output feature of the tile
+    const int nkb = P.d / BK / KS, kb0 = rank * nkb;                      // this CTA's k-blocks
+    constexpr int QL = 4 / KS;                                            // lane quarters a CTA finishes
+    uint32_t budget = WAIT_POLLS;
+    unsigned short xr[SW_UR];                                             // residual values fetched ahead (epilogue warps)
+
+    if (tid == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(tfull, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
+    HEAD_STAMP(1);
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // The weights do not depend on the stream's previous kernel: the first ring-full of weight tiles
+            // is requested before that kernel is known to be complete, the rows of X -- its output -- after.
+            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+            const int ahead = min(stages, nkb);
+            for (int kb = 0; kb < ahead; ++kb) {
+                mbar_expect_tx(full0 + 8 * kb, stage_bytes);
+                tma_load_2d(base + kb * stage_bytes, &mapW, (kb0 + kb) * BK, n0, full0 + 8 * kb);
+            }
+            HEAD_STAMP(2);
+            asm volatile("griddepcontrol.wait;" ::: "memory");
+            HEAD_STAMP(3);
+            for (int kb = 0; kb < ahead; ++kb)
+                tma_load_2d(base + kb * stage_bytes + a_bytes, &mapX, (kb0 + kb) * BK, 0, full0 + 8 * kb);
+            uint32_t stage = 0, phase = 1;                                // the ring has been filled once
+            for (int kb = ahead; kb < nkb; ++kb) {
+                mbar_wait(empty0 + 8 * stage, phase ^ 1u, P.status, budget);
+                const uint32_t a = base + stage * stage_bytes, b = a + a_bytes;
+                mbar_expect_tx(full0 + 8 * stage, stage_bytes);
+                tma_load_2d(a, &mapW, (kb0 + kb) * BK, n0, full0 + 8 * stage);     // 128 weight rows
+                tma_load_2d(b, &mapX, (kb0 + kb) * BK, 0, full0 + 8 * stage);      // the rows of X (zeros past M)
+                if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc(Npad);
+            uint32_t stage = 0, phase = 0;
+            for (int kb = 0; kb < nkb; ++kb) {
+                mbar_wait(full0 + 8 * stage, phase, P.status, budget);
+                if (kb == 0) HEAD_STAMP(2);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a = base + stage * stage_bytes, b = a + a_bytes;
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k)
+                    umma_bf16(tmem, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+                umma_commit(empty0 + 8 * stage);
+                if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+            }
+            umma_commit(tfull);
+            HEAD_STAMP(3);
+        }
+    } else {
+        // the residual values of this warp's first rows, requested while the weights stream
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const unsigned short* xcol = reinterpret_cast<const unsigned short*>(P.X) + n0 + rank * QL * 32 + lane;
+#pragma unroll
+        for (int u = 0; u < SW_UR; ++u) {
+            const int m = (warp - 2) + 4 * u;
+            xr[u] = m < P.M ? __ldg(xcol + (size_t)m * P.d) : (unsigned short)0;
+        }
+        mbar_wait(tfull, 0, P.status, budget);                            // this CTA's accumulator is complete
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        HEAD_STAMP(4);
+    }
+    __syncwarp();
+    cluster_sync_all();          // every CTA of the cluster has consumed its ring: it may now be written from outside
+    HEAD_STAMP(5);
+
+    if (warp >= 2) {
+        // lane quarter q of the accumulator goes to the CTA that finishes it
+        const int q = warp & 3, dst = q / QL, ql = q - dst * QL;
+        const uint32_t slot = smem_u32(recv) + (uint32_t)(((rank * QL + ql) * Npad) * 32 + lane) * 4u;
+        for (int c0 = 0; c0 < Npad; c0 += 32) {
+            float v[32];
+            tmem_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, v);
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (c0 + j < P.M) st_cluster_f32(slot + (uint32_t)((c0 + j) * 32) * 4u, (uint32_t)dst, v[j]);
+        }
+    }
+    HEAD_STAMP(6);
+    __syncwarp();
+    cluster_sync_all();          // all contributions have arrived
+    HEAD_STAMP(7);
+    const int ntile32 = P.d / 32;
+    if (warp >= 2) {
+        // Eight rows at a time, step by step across the eight: one warp per scheduler has nothing else to
+        // hide a row's latencies behind.  The next eight residuals are requested first.
+        const int e = warp - 2;
+        for (int ql = 0; ql < QL; ++ql) {
+            const int n = n0 + (rank * QL + ql) * 32 + lane;
+            const float bias = P.bias ? __bfloat162float(P.bias[n]) : 0.f;
+            const float wo = P.w_out ? __bfloat162float(P.w_out[n]) : 0.f;
+            const unsigned short* xcol = reinterpret_cast<const unsigned short*>(P.X) + n;
+            if (ql > 0) {
+#pragma unroll
+                for (int u = 0; u < SW_UR; ++u) {
+                    const int m = e + 4 * u;
+                    xr[u] = m < P.M ? __ldg(xcol + (size_t)m * P.d) : (unsigned short)0;
+                }
+            }
+            for (int m0 = e; m0 < P.M; m0 += 4 * SW_UR) {
+                unsigned short xn[SW_UR];
+                float z[SW_UR], y[SW_UR];
+#pragma unroll
+                for (int u = 0; u < SW_UR; ++u) {
+                    const int m = m0 + 4 * (SW_UR + u);
+                    xn[u] = m < P.M ? __ldg(xcol + (size_t)m * P.d) : (unsigned short)0;
+                }
+#pragma unroll
+                for (int u = 0; u < SW_UR; ++u) {
+                    const int m = min(m0 + 4 * u, Npad - 1);
+                    z[u] = bias;
+#pragma unroll
+                    for (int src = 0; src < KS; ++src) z[u] += recv[((src * QL + ql) * Npad + m) * 32 + lane];
+                }
+#pragma unroll
+                for (int u = 0; u < SW_UR; ++u) y[u] = __uint_as_float((uint32_t)xr[u] << 16) + silu(z[u]);
+                if (P.Y) {
+#pragma unroll
+                    for (int u = 0; u < SW_UR; ++u)
+                        if (m0 + 4 * u < P.M) P.Y[(size_t)(m0 + 4 * u) * P.d + n] = __float2bfloat16_rn(y[u]);
+                }
+                if (P.partial) {
+#pragma unroll
+                    for (int u = 0; u < SW_UR; ++u) y[u] *= wo;
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+                        for (int u = 0; u < SW_UR; ++u) y[u] += __shfl_xor_sync(0xffffffffu, y[u], o);
+#pragma unroll
+                    for (int u = 0; u < SW_UR; ++u)
+                        if (lane == u && m0 + 4 * u < P.M) P.partial[(size_t)(m0 + 4 * u) * ntile32 + (n >> 5)] = y[u];
+                }
+#pragma unroll
+                for (int u = 0; u < SW_UR; ++u) xr[u] = xn[u];
+            }
+        }
+    }
+    HEAD_STAMP(8);
+    if (P.partial) {
+        // last block: the CTA that finishes last adds every row's partial dots (a warp per row, fixed order)
+        // and applies the sigmoid
+        __shared__ int last;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) last = (atomicAdd(P.done_ctr, 1) == (int)gridDim.x - 1);
+        __syncthreads();
+        if (last) {
+            __threadfence();
+            for (int m = warp; m < P.M; m += SW_THREADS / 32) {
+                float v = 0.f;
+                for (int t = lane; t < ntile32; t += 32) v += __ldcg(P.partial + (size_t)m * ntile32 + t);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                if (lane == 0) P.accept_prob[m] = 1.f / (1.f + __expf(-(v + P.b_out)));
+            }
+            if (tid == 0) *P.done_ctr = 0;                                // ready for the next call
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    HEAD_STAMP(9);
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)tmem_cols) : "memory");
     }
 }
 
@@ -609,6 +862,65 @@ bool make_map(CUtensorMap* map, const void* ptr, int rows, int cols, int box_row
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The map of an operand, from the context's cache when this operand has been seen before.  The map is
+// copied out: the next look-up may recycle the slot it came from.
+bool cached_map(specdec_ctx* ctx, CUtensorMap* out, const void* ptr, int rows, int cols, int box_rows) {
+    static_assert(sizeof(CUtensorMap) <= sizeof(HeadMapEntry::map), "tensor map larger than its cache slot");
+    for (HeadMapEntry& e : ctx->head_maps)
+        if (e.ptr == ptr && e.rows == rows && e.cols == cols && e.box_rows == box_rows) {
+            memcpy(out, e.map, sizeof(CUtensorMap));
+            return true;
+        }
+    if (!make_map(out, ptr, rows, cols, box_rows)) return false;
+    HeadMapEntry& e = ctx->head_maps[ctx->head_map_next];
+    ctx->head_map_next = (ctx->head_map_next + 1) % 32;
+    memcpy(e.map, out, sizeof(CUtensorMap));
+    e.ptr = ptr;
+    e.rows = rows;
+    e.cols = cols;
+    e.box_rows = box_rows;
+    return true;
+}
+
+cudaError_t launch_swap(const CUtensorMap& mx, const CUtensorMap& mw, const BlockParams& p, int Npad, cudaStream_t s) {
+    const int nkb_all = p.d / BK;
+    const int KS = nkb_all % 4 == 0 ? 4 : 2;                              // d is a multiple of 128: at least two k-blocks
+    const int nkb = nkb_all / KS;
+    const int stage_bytes = BM * BK * 2 + Npad * BK * 2;
+    // Two CTAs fit on an SM when the ring stays near 100 KB: the next block's CTAs then become resident while
+    // this block's finish, and fetch their first weight tiles meanwhile.
+    const int ring_cap = 4 * stage_bytes <= 100 * 1024 ? 100 * 1024 : 200 * 1024;
+    const int stages = std::max(1, std::min(nkb, ring_cap / stage_bytes));
+    const int ring = std::max(stages * stage_bytes, 512 * Npad);
+    const int smem = ring + 1024 + 256 + 16 * stages;
+    int tmem_cols = 32;
+    while (tmem_cols < Npad) tmem_cols *= 2;
+    auto kern = KS == 4 ? head_swap_kernel<4> : head_swap_kernel<2>;
+    static unsigned long long allowed[2] = {0, 0};                        // per device: large dynamic shared memory granted
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!((allowed[KS == 4] >> (dev & 63)) & 1ull)) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        allowed[KS == 4] |= 1ull << (dev & 63);
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((p.d / BM) * KS));
+    cfg.blockDim = dim3(SW_THREADS);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)KS;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may be placed while the previous kernel drains
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kern, mx, mw, p, Npad, stages, tmem_cols);
+}
+
 template <int BN>
 cudaError_t launch_block(const CUtensorMap& mx, const CUtensorMap& mw, const BlockParams& p, cudaStream_t s) {
     cudaError_t e = cudaFuncSetAttribute(head_block_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM);
@@ -624,6 +936,14 @@ int fail(specdec_ctx* ctx, int code, const char* msg) {
 }
 
 }  // namespace
+
+#ifdef SPECDEC_STAMPS
+// Diagnostic build only (not part of the public header): the phase timestamps of one CTA of the last two
+// launches of the weights-as-M kernel, [block (0 first / 1 last)][warp][slot] in ns of the global timer.
+extern "C" int specdec_debug_head_stamps(long long* out) {
+    return (int)cudaMemcpyFromSymbol(out, head_stamps, sizeof(head_stamps));
+}
+#endif
 
 extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const specdec_head* head, int B, int K,
                                    float* accept_prob, void* stream) {
@@ -652,11 +972,14 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
     }
     // few rows (the online, one-token-per-call use): narrow column tiles so that the weight stream is
     // spread over many SMs; otherwise the widest tile the width allows
-    const int BN = M <= 256 ? 64 : (d % 256 == 0 ? 256 : 128);
+    const int BN = d % 256 == 0 ? 256 : 128;
+    // 17 to 256 rows: the weights as the M-side operand, N = the rows rounded up to 16
+    const int Npad = (int)((M + 15) / 16 * 16);
     // a handful of rows: the weight stream on the CUDA cores (no tensor maps needed)
     // 5 to 16 rows: the same stream through warp-level MMAs (X rows in shared memory: d <= 4096)
     const bool mma16_path = M > 4 && M <= MM_ROWS && d % 512 == 0 && d <= 4096;
     const bool rows_path = !mma16_path && M <= 8 && d % 256 == 0 && d <= 8192;
+    const bool swap_path = !mma16_path && !rows_path && M <= 256;
     for (int k = 0; k < D; ++k) {
         const void* W = head->W[k];
         const void* bias = head->b ? head->b[k] : nullptr;
@@ -664,7 +987,8 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
             return fail(ctx, SPECDEC_EINVAL, "accept_head: weights and biases must be non-null and 16-byte aligned");
         const bool last = (k == D - 1);
         CUtensorMap mx, mw;
-        if (!rows_path && !mma16_path && (!make_map(&mx, x, (int)M, d, BM) || !make_map(&mw, W, d, d, BN)))
+        if (!rows_path && !mma16_path && (!cached_map(ctx, &mx, x, (int)M, d, swap_path ? Npad : BM) ||
+                                          !cached_map(ctx, &mw, W, d, d, swap_path ? BM : BN)))
             return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
         BlockParams p;
         p.X = x;
@@ -677,19 +1001,19 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
         p.d = d;
         p.sm_count = ctx->sm_count;
         p.status = ctx->status;
-        p.done_ctr = ctx->task_ctl + 5;
+        p.done_ctr = ctx->task_ctl + (swap_path ? 6 : 5);
         p.accept_prob = accept_prob;
         p.b_out = head->b_out;
         cudaError_t e = mma16_path ? launch_mma16(p, s)
                         : rows_path ? (M <= 1 ? launch_rows<1>(p, s) : M <= 2 ? launch_rows<2>(p, s)
                                      : M <= 4 ? launch_rows<4>(p, s) : launch_rows<8>(p, s))
-                        : BN == 256 ? launch_block<256>(mx, mw, p, s)
-                        : BN == 128 ? launch_block<128>(mx, mw, p, s) : launch_block<64>(mx, mw, p, s);
+                        : swap_path ? launch_swap(mx, mw, p, Npad, s)
+                        : BN == 256 ? launch_block<256>(mx, mw, p, s) : launch_block<128>(mx, mw, p, s);
         if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
         ctx->launches += 1;
         x = p.Y;
     }
-    if (!rows_path && !mma16_path) {
+    if (!rows_path && !mma16_path && !swap_path) {
         head_finish_kernel<<<(int)((M + 127) / 128), 128, 0, s>>>(ctx->head_partial, (int)M, 2 * d / BN, head->b_out, accept_prob);
         ctx->launches += 1;
     }

@@ -6,6 +6,14 @@
 
 #include "specdec.h"
 
+// A tensor map (TMA descriptor) the acceptance head has built, kept so that a repeated call with the same
+// operand does not pay the driver's encoding again.
+struct HeadMapEntry {
+    const void* ptr = nullptr;
+    int rows = 0, cols = 0, box_rows = 0;
+    alignas(64) unsigned char map[128];
+};
+
 struct specdec_ctx {
     int device = 0;
     int max_B = 0, max_K = 0, max_d = 0;
@@ -18,7 +26,7 @@ struct specdec_ctx {
     uint32_t* status = nullptr;   // sticky SPECDEC_DATA_* bits
     float4* norms = nullptr;      // [max_B * (max_K+1)]  log2 normalisers {hi_p, lo_p, hi_q, lo_q} per position
     int2* tasks = nullptr;        // [max_B]              rows whose y' is still to be drawn: {b, n}
-    int32_t* task_ctl = nullptr;  // [8]                  two-launch path: {tasks, finished CTAs}; fused path: {-, -, -, head, finished}; [5]: CTAs done in the few-row head block
+    int32_t* task_ctl = nullptr;  // [8]                  two-launch path: {tasks, finished CTAs}; fused path: {-, -, -, head, finished}; [5], [6]: CTAs done in the last head block (few-row kernels, weights-as-M kernel)
     int32_t* task_ready = nullptr;// [max_B]              fused path: record {epoch:24, mode:2, n:6} of each resolved row
     uint32_t epoch = 0;
     uint64_t launches = 0;
@@ -31,6 +39,8 @@ struct specdec_ctx {
     // acceptance-head activations (device, bf16) and split-N partial logits
     void* act[2] = {nullptr, nullptr};   // [max_B*max_K, max_d] each
     float* head_partial = nullptr;       // [max_B*max_K, max_d/32]
+    HeadMapEntry head_maps[32];          // round-robin cache, keyed by (pointer, rows, cols, box rows)
+    int head_map_next = 0;
     char err[256] = "no error";
 };
 

@@ -190,7 +190,7 @@ def test_online_head_and_stop_step_replay_algorithm_1():
         want = orc.accept_head(step_hidden, list(zip(Ws, bs)), w_out, b_out)
         got = a.cpu().numpy()
         assert np.max(np.abs(got - want) / want) <= HEAD_RTOL
-        np.testing.assert_allclose(got[:, 0], batched[:, j], rtol=1e-4)
+        np.testing.assert_allclose(got[:, 0], batched[:, j], rtol=1e-3)   # two kernels, two summation orders, bf16 activations
         stop = specdec.specdec_stop_step(ctx, a.reshape(B), p_hat, h).cpu().numpy()
         o_hat, o_stop = orc.stop_step(o_hat.astype(np.float32), got[:, 0], h)
         near = np.abs(1.0 - o_hat - np.float32(h)) < parity.BOUNDARY
