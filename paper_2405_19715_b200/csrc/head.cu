@@ -900,7 +900,7 @@ cudaError_t launch_swap(const CUtensorMap& mx, const CUtensorMap& mw, const Bloc
     int dev = 0;
     cudaGetDevice(&dev);
     if (!((allowed[KS == 4] >> (dev & 63)) & 1ull)) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024);   // the opt-in limit less the static part
         if (e != cudaSuccess) return e;
         allowed[KS == 4] |= 1ull << (dev & 63);
     }
