@@ -324,12 +324,27 @@ def run_ours(args, cfg):
     from paper_2405_19715_b200 import specdec
     to_torch = specdec.from_numpy
     rank, world, local = dist_env()
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    init_dist(world, dev)
     cfg = shard_config(cfg, rank)
     inp = wl.make_verify_inputs(cfg)
     lens_np = inp["cand_len"]
+    # The oracle is timed first, before this process touches the GPU: its all-cores leg forks workers,
+    # and a process forked after CUDA has been initialised is not safe to run.
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        hd0 = wl.make_head_inputs(wl.CONFIGS["cfg5"].scaled(B=cfg.B, K=cfg.K, seed=cfg.seed))
+        rate, rows, dt = oracle_sample_rate(cfg, inp, args.cpu_budget, hd0, args.top_k or None)
+        cpu_baseline = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": f"first {rows} of {cfg.B} batch rows of {cfg.name}, {dt:.1f} s"}
+        try:
+            rate_n, rows_n, dt_n, cores = oracle_all_cores_rate(cfg, inp, args.cpu_budget, rate, hd0, args.top_k or None)
+            cpu_baseline["all_cores"] = {
+                "value": rate_n, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"first {rows_n} of {cfg.B} batch rows of {cfg.name} over {cores} forked workers, {dt_n:.1f} s"}
+        except Exception as e:                       # the single-core figure stands on its own
+            cpu_baseline["all_cores"] = {"unavailable": repr(e)}
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    init_dist(world, dev)
     es = 2 if cfg.dtype == "bf16" else 4
     per_copy = cfg.B * (2 * cfg.K + 1) * cfg.V * es
     copies = 1 if per_copy > 2 * 126e6 else int(np.ceil(2 * 126e6 / per_copy)) + 1
@@ -433,6 +448,25 @@ def run_ours(args, cfg):
                      "burst_ms_times_mhz": None if not clocks or not clocks.get("sm_mhz") else
                      {"head": head_ms * clocks["sm_mhz"], "verify": verify_ms * clocks["sm_mhz"]}}
 
+    # the same verify/correct call on ONE copy of the inputs, back to back: where a workload fits in L2 this is
+    # the warm figure (inputs served from L2), reported beside the cold one of the timed region
+    warm_ms = None
+    if copies > 1 and args.top_k == 0:
+        d0 = devs[0]
+        def warm_call():
+            specdec.specdec_verify_correct(ctx, d0["target_logits"], d0["draft_logits"], d0["cand_tokens"], d0["cand_len"],
+                                           d0["uniforms"], T, n_out, t_out, flags=args.kernel)
+        for _ in range(5):
+            warm_call()
+        wev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        torch.cuda.synchronize()
+        wev[0].record()
+        for i in range(args.steps):
+            warm_call()
+            wev[i + 1].record()
+        torch.cuda.synchronize()
+        warm_ms = float(np.mean([wev[i].elapsed_time(wev[i + 1]) for i in range(args.steps)]))
+
     # end to end through the host-buffer entry point (pinned host inputs, results back on the host)
     e2e_steps = max(1, min(args.steps, 5))
     h_n = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
@@ -482,7 +516,11 @@ def run_ours(args, cfg):
             "roofline": {"kernel": f"verify/correct ({kernel_name})", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"] + " copy bandwidth",
                          "frac_of_nominal_8TBs": achieved / 8000.0, "algorithmic_bytes": alg, "kernel_ms": verify_ms,
-                         "traffic": ncu_traffic(f"{kernel_name}<{cfg.dtype}>", units)},
+                         "traffic": ncu_traffic(f"{kernel_name}<{cfg.dtype}>", units),
+                         "cache": "cold: every step reads its logits from HBM",
+                         "warm": None if warm_ms is None else
+                         {"kernel_ms": warm_ms, "achieved": alg / (warm_ms * 1e-3) / 1e9, "unit": "GB/s",
+                          "note": "same call repeated on one copy of the inputs (served from L2 where they fit); not a DRAM figure"}},
             "parts_ms": {"head": head_ms, "stop": stop_ms, "verify": verify_ms},
             # the timed region lasts milliseconds at full clocks: the burst peak is its denominator;
             # the power-capped loop is measured against the sustained one
@@ -501,17 +539,8 @@ def run_ours(args, cfg):
         if args.top_k > 0:
             line["config"]["top_k"] = args.top_k
             line["e2e"] = None
-        if world == 1 and not args.no_cpu_baseline:
-            rate, rows, dt = oracle_sample_rate(cfg, inp, args.cpu_budget, hd, args.top_k or None)
-            line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                    "sample": f"first {rows} of {cfg.B} batch rows of {cfg.name}, {dt:.1f} s"}
-            try:
-                rate_n, rows_n, dt_n, cores = oracle_all_cores_rate(cfg, inp, args.cpu_budget, rate, hd, args.top_k or None)
-                line["cpu_baseline"]["all_cores"] = {
-                    "value": rate_n, "unit": UNIT, "cores": cores, "kind": "oracle",
-                    "sample": f"first {rows_n} of {cfg.B} batch rows of {cfg.name} over {cores} forked workers, {dt_n:.1f} s"}
-            except Exception as e:                       # the single-core figure stands on its own
-                line["cpu_baseline"]["all_cores"] = {"unavailable": repr(e)}
+        if cpu_baseline is not None:
+            line["cpu_baseline"] = cpu_baseline
         print(json.dumps(line), flush=True)
     if world > 1:
         import torch.distributed as dist
@@ -605,6 +634,44 @@ def run_phases(args, cfg):
         k = min(n - 1, int(round(f * (n - 1))))
         print(f"| {k + 1} of {n} | {sa[k]:.1f} | {da[k]:.1f} |")
     ctx.set_phase_stamps(None)
+    ctx.close()
+
+
+def run_head_phases(args):
+    """Phase timestamps of one CTA of the weights-as-M head kernel (17 to 256 rows) for one cold call of the
+    acceptance head with d = 4096, D = 2 and --batch rows (default 64): diagnostic build, not a benchmark line."""
+    import ctypes
+    from paper_2405_19715_b200 import build as libbuild, specdec
+    lib = specdec.use_library(libbuild.build(stamps=True))
+    torch.cuda.set_device(0)
+    M, d, D, copies = args.batch or 64, 4096, 2, 6
+    g = torch.Generator(device="cuda").manual_seed(1)
+    Ws = [[(torch.randn(d, d, device="cuda", generator=g) * 0.02).to(torch.bfloat16) for _ in range(D)] for _ in range(copies)]
+    w_out = (torch.randn(d, device="cuda", generator=g) * 0.02).to(torch.bfloat16)
+    ctx = specdec.Context(M, 1, max_d=d)
+    x = torch.randn(M, 1, d, device="cuda", generator=g).to(torch.bfloat16)
+    out = torch.empty(M, 1, dtype=torch.float32, device="cuda")
+    rows = []
+    for i in range(max(args.steps, 3) + 3):
+        torch.cuda.synchronize()
+        specdec.specdec_accept_head(ctx, x, Ws[i % copies], None, w_out, 0.1, out)      # weights not seen for 5 calls: cold
+        torch.cuda.synchronize()
+        buf = (ctypes.c_longlong * 192)()
+        lib.specdec_debug_head_stamps(buf)
+        a = np.array(buf[:], dtype=np.float64).reshape(2, 6, 16)[:, :, :10]
+        if i >= 3:
+            rows.append(np.where(a > 0, (a - a[a > 0].min()) * 1e-3, np.nan))
+    a = np.nanmedian(np.stack(rows), 0)
+    names = ["CTA start", "barriers, tensor memory ready", "TMA: first weight tiles requested / MMA: first stage landed",
+             "TMA: previous kernel complete, X requested / MMA: all MMAs issued", "epilogue warps: accumulator complete",
+             "cluster barrier 1 (every ring consumed)", "lane quarters sent to their owners", "cluster barrier 2 (all partial sums in)",
+             "epilogue done", "sigmoid by the last CTA (last block), CTA end"]
+    print(f"acceptance head, M={M} rows, d={d}, D={D}, cold weights, one isolated call: one CTA of each of the two launches; "
+          f"microseconds from the first CTA start, median of {len(rows)} calls")
+    print("| phase | block 1: TMA warp | MMA warp | epilogue warp | block 2: TMA warp | MMA warp | epilogue warp |\n|---|---|---|---|---|---|---|")
+    f = lambda v: "-" if np.isnan(v) else f"{v:.2f}"
+    for k, nm in enumerate(names):
+        print(f"| {nm} | {f(a[0, 0, k])} | {f(a[0, 1, k])} | {f(a[0, 2, k])} | {f(a[1, 0, k])} | {f(a[1, 1, k])} | {f(a[1, 2, k])} |")
     ctx.close()
 
 
@@ -702,6 +769,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling runs)")
     ap.add_argument("--phases", action="store_true",
                     help="print per-phase device timestamps of the one-CTA-per-unit verify/correct kernel (diagnostic build)")
+    ap.add_argument("--head-phases", action="store_true",
+                    help="print phase timestamps of the weights-as-M head kernel for --batch rows (diagnostic build)")
     ap.add_argument("--stub-step", action="store_true", help="launcher self-check: gloo ranks on the CPU, empty step")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.workload]
@@ -717,6 +786,8 @@ def main():
         sys.exit(rc)
     if args.stub_step:
         run_stub(args)
+    elif args.head_phases:
+        run_head_phases(args)
     elif args.phases:
         run_phases(args, cfg)
     elif args.vocab_shards:

@@ -293,3 +293,41 @@ def test_many_candidates_per_row(flags):
     assert rep["rows"] == 4 and c.device_status() == 0
     assert gpu["n_accepted"][0] == 80 and gpu["n_accepted"][3] >= 40
     c.close()
+
+
+def test_gpu_draws_follow_the_target_law():
+    """Secondary statistical check of the CUDA path itself: with one candidate per row drawn from q and
+    seeded uniforms, the token a row emits (the candidate when accepted, y' otherwise) must be
+    distributed as p (Appendix C).  2e5 rows at V = 8, chi-square with 7 degrees of freedom; the same
+    rows also emit p-distributed bonus tokens when every candidate is accepted (checked on the rows
+    that accept)."""
+    rng = np.random.default_rng(99)
+    V, N = 8, 200_000
+    t = rng.normal(scale=1.5, size=V).astype(np.float32)
+    d = rng.normal(scale=1.5, size=V).astype(np.float32)
+    p = np.exp(t.astype(np.float64)); p /= p.sum()
+    q = np.exp(d.astype(np.float64)); q /= q.sum()
+    ys = rng.choice(V, size=N, p=q).astype(np.int32)
+    uni = rng.random((N, 2)).astype(np.float32)
+    uni = np.minimum(uni, np.float32(1.0 - 2.0 ** -24))
+    big = specdec.Context(max_B=N, max_K=1)
+    try:
+        inp = dict(target_logits=np.broadcast_to(t, (N, 2, V)).copy(), draft_logits=np.broadcast_to(d, (N, 1, V)).copy(),
+                   cand_tokens=ys.reshape(N, 1), cand_len=None, uniforms=uni, temperature=1.0)
+        gpu = parity.run_gpu_verify(big, inp, specdec.VERIFY_DIRECT, want_stats=False)
+        assert big.device_status() == 0
+    finally:
+        big.close()
+    n, nxt = gpu["n_accepted"], gpu["next_token"]
+    emitted = np.where(n == 1, ys, nxt)
+    counts = np.bincount(emitted, minlength=V)
+    chi2 = ((counts - N * p) ** 2 / (N * p)).sum()
+    assert chi2 < 29.9, (chi2, counts)                      # P(chi2_7 > 29.9) ~ 1e-4
+    # P(accept) = sum min(p, q)
+    acc = float((n == 1).mean())
+    assert abs(acc - np.minimum(p, q).sum()) < 4.0 * np.sqrt(0.25 / N)
+    # the bonus token of the accepting rows (target row 1 = the same p) is p-distributed too
+    bonus = nxt[n == 1]
+    cb = np.bincount(bonus, minlength=V)
+    chi2b = ((cb - len(bonus) * p) ** 2 / (len(bonus) * p)).sum()
+    assert chi2b < 29.9, (chi2b, cb)
