@@ -651,6 +651,33 @@ def run_head_phases(args):
     ctx = specdec.Context(M, 1, max_d=d)
     x = torch.randn(M, 1, d, device="cuda", generator=g).to(torch.bfloat16)
     out = torch.empty(M, 1, dtype=torch.float32, device="cuda")
+    if M > 256:                                     # the 128-row-tile kernel: per-tile stamps of its first and last CTA
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        tl, ms = [], []
+        for i in range(max(args.steps, 3) + 3):
+            torch.cuda.synchronize()
+            e0.record()
+            specdec.specdec_accept_head(ctx, x, Ws[i % copies], None, w_out, 0.1, out)
+            e1.record()
+            torch.cuda.synchronize()
+            buf = (ctypes.c_longlong * 128)()
+            lib.specdec_debug_head_tile_stamps(buf)
+            a = np.array(buf[:], dtype=np.float64).reshape(2, 8, 8)[:, :, :6]
+            if i >= 3:
+                tl.append(np.where(a > 0, (a - a[a > 0].min()) * 1e-3, np.nan))
+                ms.append(e0.elapsed_time(e1))
+        a = np.nanmedian(np.stack(tl), 0)
+        print(f"acceptance head, M={M} rows, d={d}, D={D}: tiles of the LAST block's launch on its first CTA (4 tiles at M=4096) and its "
+              f"last CTA (3 tiles); microseconds from that launch's first stamp, median of {len(tl)} isolated calls; "
+              f"whole call by CUDA events {1e3 * np.mean(ms):.1f} us")
+        print("| CTA | tile | first k-block requested | accumulator free | first k-block landed | all MMAs issued | accumulator complete | epilogue done |\n|---|---|---|---|---|---|---|---|")
+        f = lambda v: "-" if np.isnan(v) else f"{v:.2f}"
+        for c in range(2):
+            for t in range(8):
+                if not np.isnan(a[c, t, 3]):
+                    print(f"| {'first' if c == 0 else 'last'} | {t} | " + " | ".join(f(a[c, t, k]) for k in range(6)) + " |")
+        ctx.close()
+        return
     rows = []
     for i in range(max(args.steps, 3) + 3):
         torch.cuda.synchronize()
