@@ -297,234 +297,6 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------
-// The same GEMM with a pair of CTAs per 256 x 256 tile (tcgen05 cta_group::2).  An SM takes in about 64 bytes
-// per clock from L2; a 128 x 256 tile needs 48 KB of operands per 512 clocks of MMAs (96 bytes per clock), so
-// the one-CTA kernel above is held to two thirds of the tensor rate by its own operand traffic (its per-tile
-// timestamps show 25 us per tile against 16.7 us of arithmetic, the same with 148 or 68 CTAs running).  Here
-// each CTA of the pair loads its 128 rows of X and only its 128 of the tile's 256 weight rows -- 32 KB per
-// k-block, 64 bytes per clock -- and one thread of the even CTA issues M = 256 MMAs that read both CTAs'
-// shared memory and write both CTAs' tensor memory.  TMA loads are per CTA (no multicast); both CTAs' loads
-// complete on the even CTA's barrier; the MMA commits are sent to the barriers of both CTAs; the odd CTA's
-// epilogue warps hand the accumulator back with arrivals on the even CTA's barrier.
-constexpr int PAIR_BN = 256;
-constexpr int PAIR_STAGES = 6;
-constexpr int PAIR_STAGE_BYTES = BM * BK * 2 + (PAIR_BN / 2) * BK * 2;    // 128 rows of X + 128 rows of W
-constexpr int PAIR_SMEM = PAIR_STAGES * PAIR_STAGE_BYTES + 1024 + 256;
-
-__device__ __forceinline__ uint32_t pair_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void pair_sync() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// TMA load by one CTA of a pair whose bytes are counted on the EVEN CTA's barrier (peer bit of the
-// barrier's cluster address cleared).
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar & 0xFEFFFFFFu) : "memory");
-}
-__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
-// Arrive on the barrier at this offset in both CTAs of the pair once the MMAs issued so far have completed.
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"((unsigned short)3) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_even_cta(uint32_t bar) {
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(bar), "r"(0u));
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
-}
-__host__ __device__ constexpr uint32_t umma_idesc_pair(int n) {           // M = 256 across the pair
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-}
-
-__global__ void __launch_bounds__(HEAD_THREADS, 1)
-head_pair_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW, const BlockParams P) {
-    constexpr int BN = PAIR_BN, STAGES = PAIR_STAGES, STAGE_BYTES = PAIR_STAGE_BYTES, A_BYTES = BM * BK * 2;
-    extern __shared__ unsigned char smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    unsigned char* aligned = smem_raw + (base - smem_u32(smem_raw));
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(aligned + STAGES * STAGE_BYTES);
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * STAGES, tfull0 = empty0 + 8 * STAGES,
-                   tempty0 = tfull0 + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int rank = (int)pair_rank();                                    // 0: issues the MMAs of the pair
-    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
-    const int nkb = P.d / BK;
-    const int ntn = P.d / BN, ntiles = ntn * ((P.M + 2 * BM - 1) / (2 * BM));
-    uint32_t budget = WAIT_POLLS;
-
-    if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full0 + 8 * s, 1);                                  // the even CTA's: one arrival with the bytes of both CTAs
-            mbar_init(empty0 + 8 * s, 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(tfull0 + 8 * b, 1);
-            mbar_init(tempty0 + 8 * b, 2 * EPI_WARPS);                    // the even CTA's: epilogue warps of both CTAs
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    if (warp == 1) {                      // the same warp of both CTAs allocates the pair's tensor memory
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)(2 * BN)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    pair_sync();                          // both CTAs' barriers exist before anything is sent to them
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
-
-    if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer (both CTAs)
-        if (lane == 0) {
-            uint32_t stage = 0, phase = 0;
-            for (int t = pair; t < ntiles; t += npairs) {
-                const int m0 = (t / ntn) * (2 * BM) + rank * BM, n0 = (t % ntn) * BN + rank * (BN / 2);
-                for (int kb = 0; kb < nkb; ++kb) {
-                    mbar_wait(empty0 + 8 * stage, phase ^ 1u, P.status, budget);
-                    const uint32_t a = base + stage * STAGE_BYTES, b = a + A_BYTES;
-                    if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * STAGE_BYTES);
-                    tma_load_2d_pair(a, &mapX, kb * BK, m0, full0 + 8 * stage);
-                    tma_load_2d_pair(b, &mapW, kb * BK, n0, full0 + 8 * stage);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ---------------------------------------------------------------- MMA issuer (even CTA only)
-        if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = umma_idesc_pair(BN);
-            uint32_t stage = 0, phase = 0, it = 0;
-            for (int t = pair; t < ntiles; t += npairs, ++it) {
-                const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
-                mbar_wait(tempty0 + 8 * buf, use ^ 1u, P.status, budget);      // both epilogues have drained this accumulator
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t acc = tmem + buf * BN;
-                for (int kb = 0; kb < nkb; ++kb) {
-                    mbar_wait(full0 + 8 * stage, phase, P.status, budget);
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a = base + stage * STAGE_BYTES, b = a + A_BYTES;
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k)
-                        umma_bf16_pair(acc, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), idesc,
-                                       (kb | k) != 0 ? 1u : 0u);
-                    umma_commit_pair(empty0 + 8 * stage);     // the stage is free in both CTAs once these MMAs have read it
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-                }
-                umma_commit_pair(tfull0 + 8 * buf);           // accumulator complete, in both CTAs
-            }
-        }
-    } else {
-        // ---------------------------------------------------------------- epilogue warps (both CTAs, own 128 rows)
-        const int q = warp & 3;
-        const int half = (warp - 2) >> 2;
-        constexpr int CH = BN / 32 / 2;
-        uint32_t it = 0;
-        for (int t = pair; t < ntiles; t += npairs, ++it) {
-            const int m0 = (t / ntn) * (2 * BM) + rank * BM, n0 = (t % ntn) * BN;
-            const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
-            const int m = m0 + q * 32 + lane;
-            const bool row_ok = m < P.M;
-            const uint4* xrow = reinterpret_cast<const uint4*>(P.X + (size_t)(row_ok ? m : 0) * P.d + n0);
-            uint4 xv[4], xn[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) xn[j] = row_ok ? __ldg(xrow + (half * CH) * 4 + j) : make_uint4(0, 0, 0, 0);
-            mbar_wait(tfull0 + 8 * buf, use, P.status, budget);
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            float dot = 0.f;
-#pragma unroll 1
-            for (int cc = 0; cc < CH; ++cc) {
-                const int c = half * CH + cc;
-                float acc[32];
-                tmem_ld32(tmem + buf * BN + ((uint32_t)(q * 32) << 16) + (uint32_t)(c * 32), acc);
-                uint4 bv[4], wv[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    xv[j] = xn[j];
-                    if (cc + 1 < CH) xn[j] = row_ok ? __ldg(xrow + (c + 1) * 4 + j) : make_uint4(0, 0, 0, 0);
-                    bv[j] = P.bias ? __ldg(reinterpret_cast<const uint4*>(P.bias + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
-                    wv[j] = P.w_out ? __ldg(reinterpret_cast<const uint4*>(P.w_out + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
-                }
-                const uint32_t* xw = reinterpret_cast<const uint32_t*>(xv);
-                const uint32_t* bw = reinterpret_cast<const uint32_t*>(bv);
-                const uint32_t* ww = reinterpret_cast<const uint32_t*>(wv);
-                uint32_t out[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float y0 = bf16lo(xw[j]) + silu(acc[2 * j] + bf16lo(bw[j]));
-                    const float y1 = bf16hi(xw[j]) + silu(acc[2 * j + 1] + bf16hi(bw[j]));
-                    dot = fmaf(y0, bf16lo(ww[j]), dot);
-                    dot = fmaf(y1, bf16hi(ww[j]), dot);
-                    const __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
-                    out[j] = *reinterpret_cast<const uint32_t*>(&pk);
-                }
-                if (P.Y && row_ok) {
-                    uint4* yrow = reinterpret_cast<uint4*>(P.Y + (size_t)m * P.d + n0 + c * 32);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) yrow[j] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
-                }
-            }
-            // this warp has read its part of the accumulator: tell the MMA issuer (in the even CTA)
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) {
-                if (rank == 0) mbar_arrive(tempty0 + 8 * buf);
-                else mbar_arrive_even_cta(tempty0 + 8 * buf);
-            }
-            if (P.partial && row_ok) P.partial[(size_t)m * (2 * ntn) + 2 * (t % ntn) + half] = dot;
-        }
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    pair_sync();                          // nothing is in flight towards the other CTA's barriers or tensor memory any more
-    if (warp == 1) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)(2 * BN)) : "memory");
-    }
-}
-
-cudaError_t launch_pair(const CUtensorMap& mx, const CUtensorMap& mw, const BlockParams& p, cudaStream_t s) {
-    static unsigned long long allowed = 0;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (!((allowed >> (dev & 63)) & 1ull)) {
-        cudaError_t e = cudaFuncSetAttribute(head_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PAIR_SMEM);
-        if (e != cudaSuccess) return e;
-        allowed |= 1ull << (dev & 63);
-    }
-    const int ntiles = (p.d / PAIR_BN) * ((p.M + 2 * BM - 1) / (2 * BM));
-    const int pairs = std::min(ntiles, p.sm_count / 2);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(2 * pairs));
-    cfg.blockDim = dim3(HEAD_THREADS);
-    cfg.dynamicSmemBytes = PAIR_SMEM;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, head_pair_kernel, mx, mw, p);
-}
-
-// ---------------------------------------------------------------------------------------------
 // The block for 17 to 256 rows (the online use of Eq. 3 for tens to hundreds of concurrent sequences):
 // the GEMM is a stream of the weights against a handful of rows, so the WEIGHTS are the M-side operand.
 // A tile is Z^T[128 output features, N rows of X] = W[128, k] * X^T[k, N]: one tcgen05.mma takes 128
@@ -1235,7 +1007,6 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
     const bool mma16_path = M > 4 && M <= MM_ROWS && d % 512 == 0 && d <= 4096;
     const bool rows_path = !mma16_path && M <= 8 && d % 256 == 0 && d <= 8192;
     const bool swap_path = !mma16_path && !rows_path && M <= 256;
-    const bool pair_path = !mma16_path && !rows_path && !swap_path && d % 256 == 0;     // a pair of CTAs per 256 x 256 tile
     for (int k = 0; k < D; ++k) {
         const void* W = head->W[k];
         const void* bias = head->b ? head->b[k] : nullptr;
@@ -1244,7 +1015,7 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
         const bool last = (k == D - 1);
         CUtensorMap mx, mw;
         if (!rows_path && !mma16_path && (!cached_map(ctx, &mx, x, (int)M, d, swap_path ? Npad : BM) ||
-                                          !cached_map(ctx, &mw, W, d, d, swap_path || pair_path ? BM : BN)))
+                                          !cached_map(ctx, &mw, W, d, d, swap_path ? BM : BN)))
             return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
         BlockParams p;
         p.X = x;
@@ -1264,7 +1035,6 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
                         : rows_path ? (M <= 1 ? launch_rows<1>(p, s) : M <= 2 ? launch_rows<2>(p, s)
                                      : M <= 4 ? launch_rows<4>(p, s) : launch_rows<8>(p, s))
                         : swap_path ? launch_swap(mx, mw, p, Npad, s)
-                        : pair_path ? launch_pair(mx, mw, p, s)
                         : BN == 256 ? launch_block<256>(mx, mw, p, s) : launch_block<128>(mx, mw, p, s);
         if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
         ctx->launches += 1;
