@@ -548,11 +548,10 @@ def run_ours(args, cfg):
 
 
 PHASES = [("CTA start -> length known", 0, 1), ("length known -> scalars requested", 1, 10),
-          ("scalars requested -> first thread's statistics done", 10, 2), ("statistics done -> CTA merged", 2, 3),
-
-          ("merged -> accept test + draw decision", 3, 4), ("  of which: warp 0 merges the warps' sums", 3, 11),
-          ("  of which: log-probabilities and ratio", 11, 12), ("  of which: flag and optional outputs stored", 12, 13),
-          ("  of which: earlier flags looked up, normalisers", 13, 4), ("decision -> seen by the CTA", 4, 5),
+          ("scalars requested -> first thread's share of the statistics pass done", 10, 2),
+          ("first thread done -> warps' sums merged by warp 0 (waits for the CTA's slowest warp)", 2, 11),
+          ("log-probabilities and ratio", 11, 12), ("flag and optional outputs stored", 12, 13),
+          ("earlier flags looked up, normalisers", 13, 4), ("decision -> seen by the CTA", 4, 5),
           ("draw: slab sums", 5, 6), ("draw: prefix, slab walk", 6, 7), ("no draw: decision -> arrival", 5, 7),
           ("arrival counted on the row", 7, 8), ("last arriver: ballot + outputs", 8, 9), ("whole unit", 0, 9)]
 
@@ -624,8 +623,7 @@ def run_phases(args, cfg):
     for name, _, _ in PHASES:
         x = np.concatenate(durs[name])
         print(f"| {name} | {len(x) // args.steps} | {q(x, 50):.2f} | {q(x, 10):.2f} | {q(x, 90):.2f} | {q(x, 100):.2f} |")
-    for name, x in (("first warp's statistics done -> last warp's", np.concatenate(skew)),
-                    ("warp 0's statistics done -> warps' sums merged by warp 0", np.concatenate(wait0))):
+    for name, x in (("first warp's statistics done -> last warp's (skew inside the CTA)", np.concatenate(skew)),):
         print(f"| {name} | {len(x) // args.steps} | {q(x, 50):.2f} | {q(x, 10):.2f} | {q(x, 90):.2f} | {q(x, 100):.2f} |")
     sa, da = np.mean(np.stack(start_at), 0), np.mean(np.stack(done_at), 0)
     n = len(sa)
