@@ -467,6 +467,49 @@ def run_ours(args, cfg):
         torch.cuda.synchronize()
         warm_ms = float(np.mean([wev[i].elapsed_time(wev[i + 1]) for i in range(args.steps)]))
 
+    # Short steps: the same launches replayed from a CUDA graph, so that no host work sits between them (with
+    # three library calls per step the host needs tens of microseconds, more than these steps take on the GPU).
+    # A graph holds one step per input copy, so the logits are as cold as in the timed region.
+    graph_times = None
+    if ms_per_step < 0.3 and args.top_k == 0 and world == 1:
+        n_g = max(copies, 8)
+
+        def head_call(i):
+            specdec.specdec_accept_head(ctx, hidden, Ws, bs, w_out, float(hd["b_out"]), head_prob)
+
+        def stop_call(i):
+            specdec.specdec_stop(ctx, head_prob, cfg.h, devs[i % copies]["cand_len"], stop_pos)
+
+        def verify_call(i):
+            d = devs[i % copies]
+            specdec.specdec_verify_correct(ctx, d["target_logits"], d["draft_logits"], d["cand_tokens"], d["cand_len"],
+                                           d["uniforms"], T, n_out, t_out, flags=args.kernel)
+
+        def replayed_ms(fn):
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(n_g):
+                    fn(i)
+            g.replay()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(5):
+                g.replay()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / (5 * n_g)
+
+        try:
+            graph_times = {"ms_per_step": replayed_ms(lambda i: step(i)),
+                           "parts_ms": {"head": replayed_ms(head_call), "stop": replayed_ms(stop_call), "verify": replayed_ms(verify_call)},
+                           "note": "launches replayed from a CUDA graph (no host in the loop); logits cold, head weights "
+                                   "as in the step (they stay in L2 between steps); each part replayed on its own"}
+        except Exception as e:                       # the event-timed figures stand on their own
+            graph_times = {"unavailable": repr(e)}
+        assert ctx.device_status() == 0
+
     # end to end through the host-buffer entry point (pinned host inputs, results back on the host)
     e2e_steps = max(1, min(args.steps, 5))
     h_n = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
@@ -522,6 +565,7 @@ def run_ours(args, cfg):
                          {"kernel_ms": warm_ms, "achieved": alg / (warm_ms * 1e-3) / 1e9, "unit": "GB/s",
                           "note": "same call repeated on one copy of the inputs (served from L2 where they fit); not a DRAM figure"}},
             "parts_ms": {"head": head_ms, "stop": stop_ms, "verify": verify_ms},
+            "graph_replay": graph_times,
             # the timed region lasts milliseconds at full clocks: the burst peak is its denominator;
             # the power-capped loop is measured against the sustained one
             "roofline_head": {"kernel": "acceptance head (2 x [M,4096]x[4096,4096] bf16 GEMM)", "bound": "tensor",
