@@ -467,6 +467,27 @@ def run_ours(args, cfg):
         torch.cuda.synchronize()
         warm_ms = float(np.mean([wev[i].elapsed_time(wev[i + 1]) for i in range(args.steps)]))
 
+    # Not the contract's path, reported beside it: the call with SPECDEC_VERIFY_EARLY_EXIT (units that start after
+    # an earlier position of their row has been rejected read nothing; outputs identical), cold inputs
+    early = None
+    if args.top_k == 0:
+        def early_call(i):
+            d = devs[i % copies]
+            specdec.specdec_verify_correct(ctx, d["target_logits"], d["draft_logits"], d["cand_tokens"], d["cand_len"],
+                                           d["uniforms"], T, n_out, t_out, flags=args.kernel | specdec.VERIFY_EARLY_EXIT)
+        for i in range(3):
+            early_call(i)
+        ctx.early_exit_count()
+        eev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        eev[0].record()
+        for i in range(args.steps):
+            early_call(i)
+            eev[i + 1].record()
+        torch.cuda.synchronize()
+        rows_unread = ctx.early_exit_count() / args.steps
+        early_ms = float(np.mean([eev[i].elapsed_time(eev[i + 1]) for i in range(args.steps)]))
+        early = {"kernel_ms": early_ms, "logit_rows_not_read_per_call": rows_unread, "kernel": ctx.last_kernel()}
+
     # Short steps: the same launches replayed from a CUDA graph, so that no host work sits between them (with
     # three library calls per step the host needs tens of microseconds, more than these steps take on the GPU).
     # A graph holds one step per input copy, so the logits are as cold as in the timed region.
@@ -566,6 +587,12 @@ def run_ours(args, cfg):
                           "note": "same call repeated on one copy of the inputs (served from L2 where they fit); not a DRAM figure"}},
             "parts_ms": {"head": head_ms, "stop": stop_ms, "verify": verify_ms},
             "graph_replay": graph_times,
+            "early_exit": None if early is None else dict(
+                early, bytes_read=alg - early["logit_rows_not_read_per_call"] * cfg.V * es,
+                achieved_read_gbs=(alg - early["logit_rows_not_read_per_call"] * cfg.V * es) / (early["kernel_ms"] * 1e-3) / 1e9,
+                tokens_per_s_verify_only=tokens_step / (early["kernel_ms"] * 1e-3),
+                note="SPECDEC_VERIFY_EARLY_EXIT: positions after a row's first rejection are not read when that rejection is "
+                     "already known; same n_accepted / next_token; not part of value, roofline or e2e above"),
             # the timed region lasts milliseconds at full clocks: the burst peak is its denominator;
             # the power-capped loop is measured against the sustained one
             "roofline_head": {"kernel": "acceptance head (2 x [M,4096]x[4096,4096] bf16 GEMM)", "bound": "tensor",

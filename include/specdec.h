@@ -71,6 +71,15 @@ typedef enum {
                                     a slice of the vocabulary, combined through distributed shared
                                     memory; picked automatically while the units fit the SMs twice   */
 
+/* May be OR-ed into the kernel selection (honoured by the one-CTA-per-unit kernel, i.e. by SPECDEC_VERIFY_AUTO on
+ * all but the smallest problems and by SPECDEC_VERIFY_DIRECT; ignored when accept_ratio or row_stats is requested):
+ * a (row, position) unit that finds, when it starts, that an earlier position of its row has already been rejected
+ * in this call reads no logits -- positions after the first rejection cannot change n_accepted or next_token
+ * (Algorithm 2 takes the minimum over the rejected positions).  Units are scheduled earliest position first, so
+ * on batches of several waves most units after a row's first rejection leave at once.  Drafted tokens are still
+ * range-checked at every position; outputs are identical with and without the bit. */
+#define SPECDEC_VERIFY_EARLY_EXIT 0x100u
+
 /*
  * Create a context on `device` able to serve calls with B <= max_B and K <= max_K.
  * Allocates the scratch used by verify/correct (per-(row,position) flags and draws,
@@ -92,6 +101,11 @@ int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits);
 
 /* Number of kernels this context has launched so far (for launch accounting). */
 uint64_t specdec_launch_count(const specdec_ctx* ctx);
+
+/* Synchronises `stream`; *logit_rows receives the number of logit rows (V elements each: two per candidate
+ * position, one for a bonus position) that units leaving early under SPECDEC_VERIFY_EARLY_EXIT did not read
+ * since the last call of this function (the counter is then cleared). */
+int specdec_early_exit_count(specdec_ctx* ctx, void* stream, uint64_t* logit_rows);
 
 /* Name of the kernel the last specdec_verify_correct / _topk call on this context launched (which
  * one SPECDEC_VERIFY_AUTO picked): a static string, "none" before the first call. */
@@ -137,7 +151,7 @@ int specdec_set_phase_stamps(specdec_ctx* ctx, uint64_t* stamps, size_t units);
  *                                  holds {lse_p, 0, 0, 0}; positions > L hold zeros
  *   resid_mass    dev out [B] f32 or NULL: sum_v (p_n - q_n)_+ at the first rejection,
  *                                  1 when every candidate was accepted
- *   flags                          SPECDEC_VERIFY_* kernel selection (0 = automatic)
+ *   flags                          SPECDEC_VERIFY_* kernel selection (0 = automatic), optionally | SPECDEC_VERIFY_EARLY_EXIT
  *
  * Logit rows at positions the method does not need (i > cand_len[b] of the target,
  * i >= cand_len[b] of the draft) are never read.  Arithmetic is fp32 (exponentials by

@@ -40,7 +40,7 @@ int check_verify_args(specdec_ctx* ctx, const void* target, const void* draft, i
     if (dtype != SPECDEC_F32 && dtype != SPECDEC_BF16) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown dtype %d", dtype);
     if (B < 1 || K < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "verify_correct: B, K, V must be >= 1 (got %d, %d, %d)", B, K, V);
     if (!(T > 0.f) || !std::isfinite(T)) return fail(ctx, SPECDEC_EINVAL, "verify_correct: temperature must be positive and finite");
-    if (flags > SPECDEC_VERIFY_CLUSTER) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown flags %u", flags);
+    if ((flags & ~SPECDEC_VERIFY_EARLY_EXIT) > SPECDEC_VERIFY_CLUSTER) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown flags %u", flags);
     if (B > ctx->max_B || K > ctx->max_K)
         return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: B=%d K=%d exceed the context (max_B=%d max_K=%d)", B, K, ctx->max_B, ctx->max_K);
     if (V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "verify_correct: V=%d above 2^22", V);
@@ -77,6 +77,8 @@ int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_
     if (e == cudaSuccess) e = cudaMalloc(&ctx->draw_mass, ndraw * sizeof(float));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->arrive, (size_t)max_B * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->status, sizeof(uint32_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->early_exits, sizeof(unsigned long long));
+    if (e == cudaSuccess) e = cudaMemset(ctx->early_exits, 0, sizeof(unsigned long long));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->norms, ndraw * sizeof(float4));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->tasks, (size_t)max_B * sizeof(int2));
     if (e == cudaSuccess) e = cudaMalloc(&ctx->task_ctl, 8 * sizeof(int32_t));
@@ -110,6 +112,7 @@ int specdec_destroy(specdec_ctx* ctx) {
     cudaFree(ctx->draw_mass);
     cudaFree(ctx->arrive);
     cudaFree(ctx->status);
+    cudaFree(ctx->early_exits);
     cudaFree(ctx->norms);
     cudaFree(ctx->tasks);
     cudaFree(ctx->task_ctl);
@@ -127,6 +130,18 @@ const char* specdec_last_error(const specdec_ctx* ctx) { return ctx ? ctx->err :
 uint64_t specdec_launch_count(const specdec_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 const char* specdec_last_kernel(const specdec_ctx* ctx) { return ctx ? ctx->last_kernel : "none"; }
+
+int specdec_early_exit_count(specdec_ctx* ctx, void* stream, uint64_t* units) {
+    if (!ctx || !units) return SPECDEC_EINVAL;
+    if (int rc = specdec_use_device(ctx)) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned long long host = 0;
+    CU(ctx, cudaMemcpyAsync(&host, ctx->early_exits, sizeof(host), cudaMemcpyDeviceToHost, s));
+    CU(ctx, cudaMemsetAsync(ctx->early_exits, 0, sizeof(host), s));
+    CU(ctx, cudaStreamSynchronize(s));
+    *units = host;
+    return SPECDEC_OK;
+}
 
 int specdec_set_phase_stamps(specdec_ctx* ctx, uint64_t* stamps, size_t units) {
     if (!ctx) return SPECDEC_EINVAL;
@@ -200,7 +215,8 @@ int specdec_verify_correct(specdec_ctx* ctx, const void* target_logits, const vo
     if (ctx->stamps && (size_t)B * (K + 1) <= ctx->stamps_units) p.stamps = ctx->stamps;
 
     const bool stream_ok = verify_stream_supported(p, dtype);
-    uint32_t kind = flags;
+    uint32_t kind = flags & ~SPECDEC_VERIFY_EARLY_EXIT;
+    if ((flags & SPECDEC_VERIFY_EARLY_EXIT) && !accept_ratio && !row_stats) p.early_exits = ctx->early_exits;
     if (kind == SPECDEC_VERIFY_AUTO) {
         // One CTA per unit (four 256-thread CTAs per SM on large grids) measured at or ahead of the
         // persistent TMA pipelines at every size tried, so those stay selectable but are not picked here.

@@ -24,6 +24,7 @@ struct specdec_ctx {
     float* draw_mass = nullptr;   // [max_B * (max_K+1)]  mass of the weights that draw came from
     int32_t* arrive = nullptr;    // [max_B]              positions of a row that have finished
     uint32_t* status = nullptr;   // sticky SPECDEC_DATA_* bits
+    unsigned long long* early_exits = nullptr;   // logit rows not read by units that left early (SPECDEC_VERIFY_EARLY_EXIT) since last read
     float4* norms = nullptr;      // [max_B * (max_K+1)]  log2 normalisers {hi_p, lo_p, hi_q, lo_q} per position
     int2* tasks = nullptr;        // [max_B]              rows whose y' is still to be drawn: {b, n}
     int32_t* task_ctl = nullptr;  // [8]                  two-launch path: {tasks, finished CTAs}; fused path: {-, -, -, head, finished}; [5], [6]: CTAs done in the last head block (few-row kernels, weights-as-M kernel)
@@ -67,6 +68,7 @@ struct VerifyParams {
     int32_t* task_ctl;
     int32_t* task_ready;
     uint32_t epoch;
+    unsigned long long* early_exits = nullptr;   // non-null: units after a row's known first rejection read nothing
     unsigned long long* stamps = nullptr;   // phase timestamps, SPECDEC_STAMP_SLOTS {globaltimer ns, SM clock} pairs per unit (diagnostic builds)
 };
 

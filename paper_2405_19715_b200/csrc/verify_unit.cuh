@@ -32,6 +32,16 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
     u.L = P.lens ? ld_early_s32(P.lens + u.b) : P.K;
     int y = 0;
     if (tid == 0 && u.i < P.K) y = ld_early_s32(P.tokens + (size_t)u.b * P.K + u.i);
+    // Early exit (optional): the accept flags of the row's earlier positions are asked for in the same round
+    // trip.  If one of them already says "rejected" in this call, this position cannot be the first rejection
+    // and nothing it could compute can reach the outputs.
+    bool earlier_rejected = false;
+    if (P.early_exits && warp == 0 && u.i > 0)
+        for (int j0 = 0; j0 < u.i; j0 += 32) {
+            const int j = j0 + lane;
+            const int f = j < u.i ? ld_relaxed(P.flags + (size_t)u.b * P.K + j) : 0;   // other CTAs write these during the launch
+            earlier_rejected |= ((uint32_t)f >> 2) == P.epoch && (f & 3) >= FLAG_REJECT;
+        }
     if (u.L < 0 || u.L > P.K) {                  // bad length: the row reports -1, nothing is read
         if (u.i == 0 && tid == 0) {
             atomicOr(P.status, SPECDEC_DATA_BAD_LENGTH);
@@ -44,6 +54,27 @@ __device__ __forceinline__ void direct_unit(const VerifyParams& P, float* __rest
     if (u.i > u.L) return;
     u.bonus = (u.i == u.L);
     if (tid == 0) stamp(P, unit, 1);
+    if (P.early_exits && u.i > 0) {              // CTA-uniform decision
+        if (warp == 0) {
+            const bool any = __any_sync(0xffffffffu, earlier_rejected);
+            if (lane == 0) sh.need_draw = any;
+        }
+        __syncthreads();
+        const bool leave = sh.need_draw != 0;
+        __syncthreads();                         // sh.need_draw is written again below
+        if (leave) {
+            if (warp == 0) {
+                if (lane == 0) {                 // the drafted token is still range-checked; the flag is this call's
+                    const bool y_bad = !u.bonus && (y < 0 || y >= P.V);
+                    if (y_bad) atomicOr(P.status, SPECDEC_DATA_BAD_TOKEN);
+                    if (!u.bonus) st_relaxed(&P.flags[(size_t)u.b * P.K + u.i], (int)((P.epoch << 2) | (uint32_t)(y_bad ? FLAG_BAD : 0)));
+                    atomicAdd(P.early_exits, u.bonus ? 1ull : 2ull);      // logit rows this unit did not read
+                }
+                unit_finish(P, u, 0, -1, 0.f, lane, unit);
+            }
+            return;
+        }
+    }
 
     const size_t V = (size_t)P.V;
     const T* trow = static_cast<const T*>(P.target) + ((size_t)u.b * (P.K + 1) + u.i) * V;

@@ -331,3 +331,45 @@ def test_gpu_draws_follow_the_target_law():
     cb = np.bincount(bonus, minlength=V)
     chi2b = ((cb - len(bonus) * p) ** 2 / (len(bonus) * p)).sum()
     assert chi2b < 29.9, (chi2b, cb)
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg5"])
+def test_early_exit_leaves_the_outputs_unchanged(name):
+    """SPECDEC_VERIFY_EARLY_EXIT: units that start after an earlier position of their row has been rejected
+    read nothing.  n_accepted and next_token must be what the oracle says (and what the call without the bit
+    gives), bad tokens after the first rejection must still be reported, and on a batch of several waves a
+    good share of the units must indeed have left early."""
+    cfg = wl.CONFIGS[name]
+    inp = wl.make_verify_inputs(cfg)
+    c = specdec.Context(cfg.B, cfg.K)
+    try:
+        base = parity.run_gpu_verify(c, inp, specdec.VERIFY_DIRECT, want_stats=False)
+        c.early_exit_count()
+        fast = parity.run_gpu_verify(c, inp, specdec.VERIFY_DIRECT | specdec.VERIFY_EARLY_EXIT, want_stats=False)
+        left = c.early_exit_count()
+        assert c.device_status() == 0
+        assert np.array_equal(base["n_accepted"], fast["n_accepted"])
+        assert np.array_equal(base["next_token"], fast["next_token"])
+        rep = parity.classify_rows(inp, fast, dtype="f32", check_probs=False)
+        assert rep["exact"] + rep["boundary_n"] + rep["boundary_token"] == cfg.B
+        units = int((inp["cand_len"].astype(np.int64) + 1).sum())
+        rows = int((2 * inp["cand_len"].astype(np.int64) + 1).sum())
+        print(name, "units", units, "logit rows", rows, "rows not read", left)
+        assert 0 <= left < rows
+        if name == "cfg5":
+            assert left > rows // 4                   # 3.7 waves, earliest positions first
+        # with the optional outputs requested the bit is ignored: all positions are computed
+        full = parity.run_gpu_verify(c, inp, specdec.VERIFY_DIRECT | specdec.VERIFY_EARLY_EXIT, want_stats=True)
+        assert c.early_exit_count() == 0
+        parity.classify_rows(inp, full, dtype="f32")
+        # a bad token behind the first rejection is still seen
+        bad = dict(inp)
+        bad["cand_tokens"] = inp["cand_tokens"].copy()
+        b = int(np.argmax((base["n_accepted"] + 1 < inp["cand_len"])))      # a row with a position after its first rejection
+        if base["n_accepted"][b] + 1 < inp["cand_len"][b]:
+            bad["cand_tokens"][b, inp["cand_len"][b] - 1] = cfg.V + 5
+            out = parity.run_gpu_verify(c, bad, specdec.VERIFY_DIRECT | specdec.VERIFY_EARLY_EXIT, want_stats=False)
+            assert c.device_status() & specdec.DATA_BAD_TOKEN
+            assert out["n_accepted"][b] == -1 and out["next_token"][b] == -1
+    finally:
+        c.close()
