@@ -37,3 +37,25 @@ def test_product_path_does_not_import_the_oracle():
         if f.suffix in (".py", ".cu", ".cuh", ".h"):
             assert not re.search(r"^\s*(from|import)\s+oracle|oracle/|#include.*oracle", f.read_text(), flags=re.M), f
     assert "paper_2405_19715_b200" not in (ROOT / "oracle" / "specdec_oracle.py").read_text()
+
+
+def test_every_context_entry_point_makes_the_contexts_gpu_current():
+    """Source-level check of the rule stated in specdec.h: every exported call that takes a context and touches
+    the GPU selects the context's device first (directly or through its argument checker)."""
+    csrc = ROOT / "paper_2405_19715_b200" / "csrc"
+    text = "\n".join((csrc / f).read_text() for f in ("api.cu", "head.cu"))
+    exempt = {"specdec_create", "specdec_destroy", "specdec_last_error", "specdec_launch_count", "specdec_last_kernel",
+              "specdec_set_phase_stamps", "specdec_use_device", "specdec_verify_correct_topk_forward"}
+    found = 0
+    for m in re.finditer(r"^(?:extern \"C\" )?(?:int|uint64_t|const char\*) (specdec_[a-z_]+)\(([^)]*)\)\s*\{", text, flags=re.M):
+        name, args = m.group(1), m.group(2)
+        if name in exempt or "specdec_ctx* ctx" not in args:
+            continue
+        depth, i = 1, m.end()
+        while depth and i < len(text):
+            depth += {"{": 1, "}": -1}.get(text[i], 0)
+            i += 1
+        body = text[m.end():i]
+        assert re.search(r"specdec_use_device\(ctx\)|check_verify_args\(ctx|check_shard_args\(ctx|specdec_verify_correct\(ctx", body), name
+        found += 1
+    assert found >= 12
