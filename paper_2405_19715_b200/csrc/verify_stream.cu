@@ -176,10 +176,78 @@ __device__ __forceinline__ void produce_unit(StreamShared& ss, uint32_t ring, co
     }
 }
 
+// The statistics warps' walk over the CTA's units: every thread keeps the vectors of a tile in registers,
+// the warp-uniform reference follows the tile maxima, and at the end of a unit each warp posts its partial
+// {reference, sum} of both rows into a hand-off slot for the epilogue warps.  `stage` / `phase` are the
+// warp's place in the ring and stay valid for whatever the caller streams next.
+template <typename T>
+__device__ __forceinline__ void stats_workers(const VerifyParams& P, StreamShared& ss, uint32_t ring, uint32_t row_bytes,
+                                              int ntiles, int ncand, int tid, int lane, int warp, uint32_t& stage,
+                                              uint32_t& phase) {
+    constexpr int NP = Elem<T>::EPV / 2;
+    int k = 0;
+    Unit un;
+    uint32_t seq = 0;
+    while (next_unit(P, ss.cand_L, k, ncand, un, false)) {
+        Acc2 ap = acc2_init(), aq = acc2_init();
+        for (int t = 0; t < ntiles; ++t) {
+            const uint32_t bytes = min((uint32_t)TILE_BYTES, row_bytes - (uint32_t)t * TILE_BYTES);
+            const int nvec = bytes >> 4;
+            const uint32_t base = ring + stage * (2 * TILE_BYTES);
+            mbar_wait_warp(smem_u32(&ss.full[stage]), phase, P.status, lane);
+            // the tile's vectors of this thread, padded with -inf beyond the row's end
+            uint4 rt[ITERS], rd[ITERS];
+            float mt = -INFINITY, md = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < ITERS; ++j) {
+                const int v = tid + j * NST;
+                const uint32_t ninf = neg_inf_word(T());
+                rt[j] = rd[j] = make_uint4(ninf, ninf, ninf, ninf);
+                if (v < nvec) {
+                    rt[j] = lds128(base + v * 16);
+                    if (!un.bonus) rd[j] = lds128(base + TILE_BYTES + v * 16);
+                }
+                mt = fmaxf(mt, vec_max(rt[j], T()));
+                md = fmaxf(md, vec_max(rd[j], T()));
+            }
+            acc2_reference(ap, mt, P.c);
+            if (!un.bonus) acc2_reference(aq, md, P.c);
+            const f2 c2 = pack2(P.c, P.c);
+            const f2 np2 = pack2(-ap.rs, -ap.rs), nq2 = pack2(-aq.rs, -aq.rs);
+#pragma unroll
+            for (int j = 0; j < ITERS; ++j) {
+                f2 xt[NP], xd[NP];
+                to_pairs(rt[j], xt, T());
+                acc2_add<NP>(ap, xt, c2, np2);
+                if (!un.bonus) {
+                    to_pairs(rd[j], xd, T());
+                    acc2_add<NP>(aq, xd, c2, nq2);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ss.empty[stage]));
+            if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        // hand the unit's partial sums to the epilogue warps and move on
+        Acc fp = acc2_fold(ap), fq = acc2_fold(aq);      // rs is warp-uniform: add the lanes
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            fp.s += __shfl_xor_sync(0xffffffffu, fp.s, o);
+            fq.s += __shfl_xor_sync(0xffffffffu, fq.s, o);
+        }
+        const uint32_t slot = seq % QSLOTS, use = seq / QSLOTS;
+        if (lane == 0) {
+            if (use > 0) mbar_wait(smem_u32(&ss.slot_empty[slot]), (use - 1) & 1u, P.status);
+            ss.slots[slot][warp] = make_float4(fp.rs, fp.s, fq.rs, fq.s);
+            mbar_arrive(smem_u32(&ss.slot_full[slot]));
+        }
+        ++seq;
+        ++k;
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(STREAM_THREADS, 1) verify_stream_stats_kernel(const VerifyParams P) {
-    constexpr int N = Elem<T>::EPV;
-    constexpr int NP = N / 2;
     extern __shared__ __align__(1024) unsigned char smem[];
     StreamShared& ss = *reinterpret_cast<StreamShared*>(smem + RING_BYTES);
     const uint32_t ring = smem_u32(smem);
@@ -216,63 +284,8 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) verify_stream_stats_kernel(
 
     if (warp < NS) {
         // ------------------------------------------------------------------ worker warps
-        uint32_t stage = 0, phase = 0, seq = 0;
-        while (next_unit(P, ss.cand_L, k, ncand, un, false)) {
-            Acc2 ap = acc2_init(), aq = acc2_init();
-            for (int t = 0; t < ntiles; ++t) {
-                const uint32_t bytes = min((uint32_t)TILE_BYTES, row_bytes - (uint32_t)t * TILE_BYTES);
-                const int nvec = bytes >> 4;
-                const uint32_t base = ring + stage * (2 * TILE_BYTES);
-                mbar_wait_warp(smem_u32(&ss.full[stage]), phase, P.status, lane);
-                // the tile's vectors of this thread, padded with -inf beyond the row's end
-                uint4 rt[ITERS], rd[ITERS];
-                float mt = -INFINITY, md = -INFINITY;
-#pragma unroll
-                for (int j = 0; j < ITERS; ++j) {
-                    const int v = tid + j * NST;
-                    const uint32_t ninf = neg_inf_word(T());
-                    rt[j] = rd[j] = make_uint4(ninf, ninf, ninf, ninf);
-                    if (v < nvec) {
-                        rt[j] = lds128(base + v * 16);
-                        if (!un.bonus) rd[j] = lds128(base + TILE_BYTES + v * 16);
-                    }
-                    mt = fmaxf(mt, vec_max(rt[j], T()));
-                    md = fmaxf(md, vec_max(rd[j], T()));
-                }
-                acc2_reference(ap, mt, P.c);
-                if (!un.bonus) acc2_reference(aq, md, P.c);
-                const f2 c2 = pack2(P.c, P.c);
-                const f2 np2 = pack2(-ap.rs, -ap.rs), nq2 = pack2(-aq.rs, -aq.rs);
-#pragma unroll
-                for (int j = 0; j < ITERS; ++j) {
-                    f2 xt[NP], xd[NP];
-                    to_pairs(rt[j], xt, T());
-                    acc2_add<NP>(ap, xt, c2, np2);
-                    if (!un.bonus) {
-                        to_pairs(rd[j], xd, T());
-                        acc2_add<NP>(aq, xd, c2, nq2);
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ss.empty[stage]));
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-            }
-            // hand the unit's partial sums to the epilogue warps and move on
-            Acc fp = acc2_fold(ap), fq = acc2_fold(aq);      // rs is warp-uniform: add the lanes
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                fp.s += __shfl_xor_sync(0xffffffffu, fp.s, o);
-                fq.s += __shfl_xor_sync(0xffffffffu, fq.s, o);
-            }
-            const uint32_t slot = seq % QSLOTS, use = seq / QSLOTS;
-            if (lane == 0) {
-                if (use > 0) mbar_wait(smem_u32(&ss.slot_empty[slot]), (use - 1) & 1u, P.status);
-                ss.slots[slot][warp] = make_float4(fp.rs, fp.s, fq.rs, fq.s);
-                mbar_arrive(smem_u32(&ss.slot_full[slot]));
-            }
-            ++seq;
-            ++k;
-        }
+        uint32_t stage = 0, phase = 0;
+        stats_workers<T>(P, ss, ring, row_bytes, ntiles, ncand, tid, lane, warp, stage, phase);
         return;
     }
 
@@ -521,7 +534,6 @@ __device__ __forceinline__ bool next_unit_fused(const VerifyParams& P, const int
 template <typename T>
 __global__ void __launch_bounds__(STREAM_THREADS, 1) verify_fused_kernel(const VerifyParams P) {
     constexpr int N = Elem<T>::EPV;
-    constexpr int NP = N / 2;
     extern __shared__ __align__(1024) unsigned char smem[];
     FusedShared& fs = *reinterpret_cast<FusedShared*>(smem + RING_BYTES);
     StreamShared& ss = fs.st;
@@ -605,61 +617,8 @@ __global__ void __launch_bounds__(STREAM_THREADS, 1) verify_fused_kernel(const V
 
     if (warp < NS) {
         // ================================================================== worker warps
-        uint32_t stage = 0, phase = 0, seq = 0;
-        while (next_unit(P, ss.cand_L, k, ncand, un, false)) {
-            Acc2 ap = acc2_init(), aq = acc2_init();
-            for (int t = 0; t < ntiles; ++t) {
-                const uint32_t bytes = min((uint32_t)TILE_BYTES, row_bytes - (uint32_t)t * TILE_BYTES);
-                const int nvec = bytes >> 4;
-                const uint32_t base = ring + stage * (2 * TILE_BYTES);
-                mbar_wait_warp(smem_u32(&ss.full[stage]), phase, P.status, lane);
-                uint4 rt[ITERS], rd[ITERS];
-                float mt = -INFINITY, md = -INFINITY;
-#pragma unroll
-                for (int j = 0; j < ITERS; ++j) {
-                    const int v = tid + j * NST;
-                    const uint32_t ninf = neg_inf_word(T());
-                    rt[j] = rd[j] = make_uint4(ninf, ninf, ninf, ninf);
-                    if (v < nvec) {
-                        rt[j] = lds128(base + v * 16);
-                        if (!un.bonus) rd[j] = lds128(base + TILE_BYTES + v * 16);
-                    }
-                    mt = fmaxf(mt, vec_max(rt[j], T()));
-                    md = fmaxf(md, vec_max(rd[j], T()));
-                }
-                acc2_reference(ap, mt, P.c);
-                if (!un.bonus) acc2_reference(aq, md, P.c);
-                const f2 c2 = pack2(P.c, P.c);
-                const f2 np2 = pack2(-ap.rs, -ap.rs), nq2 = pack2(-aq.rs, -aq.rs);
-#pragma unroll
-                for (int j = 0; j < ITERS; ++j) {
-                    f2 xt[NP], xd[NP];
-                    to_pairs(rt[j], xt, T());
-                    acc2_add<NP>(ap, xt, c2, np2);
-                    if (!un.bonus) {
-                        to_pairs(rd[j], xd, T());
-                        acc2_add<NP>(aq, xd, c2, nq2);
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ss.empty[stage]));
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
-            }
-            Acc fp = acc2_fold(ap), fq = acc2_fold(aq);      // rs is warp-uniform: add the lanes
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                fp.s += __shfl_xor_sync(0xffffffffu, fp.s, o);
-                fq.s += __shfl_xor_sync(0xffffffffu, fq.s, o);
-            }
-            const uint32_t slot = seq % QSLOTS, use = seq / QSLOTS;
-            if (lane == 0) {
-                if (use > 0) mbar_wait(smem_u32(&ss.slot_empty[slot]), (use - 1) & 1u, P.status);
-                ss.slots[slot][warp] = make_float4(fp.rs, fp.s, fq.rs, fq.s);
-                mbar_arrive(smem_u32(&ss.slot_full[slot]));
-            }
-            ++seq;
-            ++k;
-        }
+        uint32_t stage = 0, phase = 0;
+        stats_workers<T>(P, ss, ring, row_bytes, ntiles, ncand, tid, lane, warp, stage, phase);
         // ---- phase 2: draw units, described by the producer's descriptors
         for (uint32_t seq2 = 0;; ++seq2) {
             mbar_wait_warp(smem_u32(&ss.full[stage]), phase, P.status, lane);     // first tile (or the end marker)
