@@ -17,6 +17,7 @@
 #include <cstring>
 
 #include "specdec_internal.h"
+#include "verify_device.cuh"
 
 namespace {
 
@@ -555,18 +556,10 @@ head_swap_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
 // in flight per lane), every row of X is read from shared memory once per four columns, and the
 // per-lane partial sums are reduced with shuffles.  The epilogue is the one of the tensor path.
 // packed fp32 pairs: one instruction, two multiply-adds (the two halves are two output columns)
-using f2 = unsigned long long;
-__device__ __forceinline__ f2 pack2(float a, float b) {
-    f2 r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-    return r;
-}
-__device__ __forceinline__ void unpack2(f2 v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
-__device__ __forceinline__ f2 fma2(f2 a, f2 b, f2 c) {
-    f2 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
+using sd::f2;
+using sd::fma2;
+using sd::pack2;
+using sd::unpack2;
 
 constexpr int GV_WARPS = 8, GV_COLS = 4, GV_UNROLL = 4;
 constexpr int GV_THREADS = GV_WARPS * 32, GV_TILE = GV_WARPS * GV_COLS;
