@@ -451,7 +451,7 @@ def run_ours(args, cfg):
     # the same verify/correct call on ONE copy of the inputs, back to back: where a workload fits in L2 this is
     # the warm figure (inputs served from L2), reported beside the cold one of the timed region
     warm_ms = None
-    if copies > 1 and args.top_k == 0:
+    if copies > 1 and args.top_k == 0 and not args.no_extras:
         d0 = devs[0]
         def warm_call():
             specdec.specdec_verify_correct(ctx, d0["target_logits"], d0["draft_logits"], d0["cand_tokens"], d0["cand_len"],
@@ -470,7 +470,7 @@ def run_ours(args, cfg):
     # Not the contract's path, reported beside it: the call with SPECDEC_VERIFY_EARLY_EXIT (units that start after
     # an earlier position of their row has been rejected read nothing; outputs identical), cold inputs
     early = None
-    if args.top_k == 0:
+    if args.top_k == 0 and not args.no_extras:
         def early_call(i):
             d = devs[i % copies]
             specdec.specdec_verify_correct(ctx, d["target_logits"], d["draft_logits"], d["cand_tokens"], d["cand_len"],
@@ -492,7 +492,7 @@ def run_ours(args, cfg):
     # three library calls per step the host needs tens of microseconds, more than these steps take on the GPU).
     # A graph holds one step per input copy, so the logits are as cold as in the timed region.
     graph_times = None
-    if ms_per_step < 0.3 and args.top_k == 0 and world == 1:
+    if ms_per_step < 0.3 and args.top_k == 0 and world == 1 and not args.no_extras:
         n_g = max(copies, 8)
 
         def head_call(i):
@@ -862,6 +862,8 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=10.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the legs outside the timed region: warm figure, early exit, graph replay (profiling runs)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (profiling runs)")
     ap.add_argument("--phases", action="store_true",
                     help="print per-phase device timestamps of the one-CTA-per-unit verify/correct kernel (diagnostic build)")
