@@ -37,7 +37,7 @@ def _run_head(ctx, hidden, Ws, bs, w_out, b_out):
 @pytest.mark.parametrize("with_bias", [False, True])
 @pytest.mark.parametrize("rows", [(7, 23), (9, 33)], ids=["161rows", "297rows"])
 def test_head_small_shapes(d, depth, with_bias, rows):
-    B, K = rows                       # 161 rows use the narrow 64-column tiles, 297 rows the 128/256-column ones;
+    B, K = rows                       # 161 rows use the weights-as-M kernel, 297 rows the 128 x 128/256 tiles;
                                       # both leave a ragged last row tile
     ctx = specdec.Context(B, K, max_d=d)
     hidden, Ws, bs, w_out, b_out = _head_problem(100 + d + depth, B, K, d, depth, with_bias)
@@ -170,7 +170,7 @@ def test_head_up_to_256_rows_at_full_width(rows):
 
 
 def test_online_head_and_stop_step_replay_algorithm_1():
-    """Algorithm 1's loop, one drafted token per call: head on [B,1,d] (narrow-tile GEMM), then
+    """Algorithm 1's loop, one drafted token per call: head on [B,1,d] (few-row / weights-as-M kernels), then
     specdec_stop_step.  Each step is checked against the oracle; the replay must also reproduce the
     batched head + stop rule."""
     B, K, d = 96, 6, 512
