@@ -92,6 +92,17 @@ def test_config4_full_size_every_row(ctx, cfg4_problem, flags):
     # rows whose drafted tokens carry +12 on the target are accepted almost surely
     peaked = np.nonzero(inp["peaked"])[0]
     assert (gpu["n_accepted"][peaked] == cfg.K).mean() > 0.8
+    if flags == specdec.VERIFY_DIRECT:
+        # the same launch with the early exit: identical n and y' on all 256 rows, and (7 waves, earliest
+        # positions first) a large share of the logit rows left unread
+        ctx.early_exit_count()
+        fast = parity.run_gpu_verify(ctx, inp, flags | specdec.VERIFY_EARLY_EXIT, want_stats=False)
+        unread = ctx.early_exit_count()
+        assert ctx.device_status() == 0
+        assert np.array_equal(fast["n_accepted"], gpu["n_accepted"]) and np.array_equal(fast["next_token"], gpu["next_token"])
+        rows = int((2 * inp["cand_len"].astype(np.int64) + 1).sum())
+        print("cfg4 early exit: logit rows not read", unread, "of", rows)
+        assert rows // 4 < unread < rows
 
 
 @pytest.mark.parametrize("flags", KERNELS, ids=KERNEL_IDS)
