@@ -14,10 +14,10 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "specdec_internal.h"
-#include "verify_device.cuh"
 
 namespace {
 
@@ -120,7 +120,7 @@ struct BlockParams {
     int M, d;
     int sm_count;
     uint32_t* status;
-    // few-row path, last block: the CTA that finishes last adds the partial dots and applies the sigmoid
+    // weights-as-M kernel, last block: the CTA that finishes last adds the partial dots and applies the sigmoid
     int32_t* done_ctr;
     float* accept_prob;
     float b_out;
@@ -298,7 +298,8 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------
-// The block for 17 to 256 rows (the online use of Eq. 3 for tens to hundreds of concurrent sequences):
+// The block for up to 256 rows (the online use of Eq. 3 in Algorithm 1's loop: one drafted token per call for one
+// to hundreds of concurrent sequences):
 // the GEMM is a stream of the weights against a handful of rows, so the WEIGHTS are the M-side operand.
 // A tile is Z^T[128 output features, N rows of X] = W[128, k] * X^T[k, N]: one tcgen05.mma takes 128
 // weight rows whatever the number of rows of X (N = M rounded up to 16); the accumulator holds one
@@ -548,277 +549,6 @@ head_swap_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// The block for a few rows (Algorithm 1 runs the head once per drafted token: M = number of
-// sequences).  With M <= 8 the block is a stream of the 2 d^2 weight bytes against rows that fit in
-// shared memory, so it runs on the CUDA cores at HBM rate: a CTA owns 32 output columns, each of
-// its 8 warps 4 of them; lanes walk along k (coalesced 512-byte pieces of a weight row, 16 of them
-// in flight per lane), every row of X is read from shared memory once per four columns, and the
-// per-lane partial sums are reduced with shuffles.  The epilogue is the one of the tensor path.
-// packed fp32 pairs: one instruction, two multiply-adds (the two halves are two output columns)
-using sd::f2;
-using sd::fma2;
-using sd::pack2;
-using sd::unpack2;
-
-constexpr int GV_WARPS = 8, GV_COLS = 4, GV_UNROLL = 4;
-constexpr int GV_THREADS = GV_WARPS * 32, GV_TILE = GV_WARPS * GV_COLS;
-
-template <int MR>                  // rows held (a power of two >= M); missing rows are zero
-__global__ void __launch_bounds__(GV_THREADS) head_rows_kernel(const BlockParams P) {
-    extern __shared__ uint4 xs[];                      // [MR][d / 8]: the rows of X, bf16
-    __shared__ float dots[GV_WARPS][MR];
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int d = P.d, dv = d >> 3, nchunk = d >> 8;   // a chunk: 256 k-elements, one 16-byte vector per lane
-    const int n0 = blockIdx.x * GV_TILE + warp * GV_COLS;
-    const uint4* wrow[GV_COLS];
-#pragma unroll
-    for (int c = 0; c < GV_COLS; ++c) wrow[c] = reinterpret_cast<const uint4*>(P.W + (size_t)(n0 + c) * d) + lane;
-
-    // first round of weight loads, then the rows of X while those are in flight
-    uint4 wv[GV_UNROLL][GV_COLS];
-#pragma unroll
-    for (int u = 0; u < GV_UNROLL; ++u)
-#pragma unroll
-        for (int c = 0; c < GV_COLS; ++c) wv[u][c] = u < nchunk ? __ldcs(wrow[c] + u * 32) : make_uint4(0, 0, 0, 0);
-    for (int i = tid; i < MR * dv; i += GV_THREADS) {
-        const int m = i / dv;
-        xs[i] = m < P.M ? __ldg(reinterpret_cast<const uint4*>(P.X) + (size_t)m * dv + (i - m * dv)) : make_uint4(0, 0, 0, 0);
-    }
-    __syncthreads();
-
-    f2 acc2[GV_COLS / 2][MR];                          // columns (2p, 2p + 1) side by side
-#pragma unroll
-    for (int p = 0; p < GV_COLS / 2; ++p)
-#pragma unroll
-        for (int m = 0; m < MR; ++m) acc2[p][m] = pack2(0.f, 0.f);
-    for (int ch0 = 0; ch0 < nchunk; ch0 += GV_UNROLL) {
-        uint4 cur[GV_UNROLL][GV_COLS];
-#pragma unroll
-        for (int u = 0; u < GV_UNROLL; ++u)
-#pragma unroll
-            for (int c = 0; c < GV_COLS; ++c) {
-                cur[u][c] = wv[u][c];
-                const int nx = ch0 + GV_UNROLL + u;    // the next round, issued before this one is consumed
-                wv[u][c] = nx < nchunk ? __ldcs(wrow[c] + nx * 32) : make_uint4(0, 0, 0, 0);
-            }
-#pragma unroll
-        for (int u = 0; u < GV_UNROLL; ++u) {
-            if (ch0 + u >= nchunk) break;
-            f2 wp[GV_COLS / 2][8];
-#pragma unroll
-            for (int p = 0; p < GV_COLS / 2; ++p) {
-                const uint32_t* wa = reinterpret_cast<const uint32_t*>(&cur[u][2 * p]);
-                const uint32_t* wb = reinterpret_cast<const uint32_t*>(&cur[u][2 * p + 1]);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    wp[p][2 * j] = pack2(bf16lo(wa[j]), bf16lo(wb[j]));
-                    wp[p][2 * j + 1] = pack2(bf16hi(wa[j]), bf16hi(wb[j]));
-                }
-            }
-#pragma unroll
-            for (int m = 0; m < MR; ++m) {
-                const uint4 xv = xs[m * dv + (ch0 + u) * 32 + lane];
-                const uint32_t* x32 = reinterpret_cast<const uint32_t*>(&xv);
-                float xf[8];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) { xf[2 * j] = bf16lo(x32[j]); xf[2 * j + 1] = bf16hi(x32[j]); }
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const f2 xx = pack2(xf[j], xf[j]);
-#pragma unroll
-                    for (int p = 0; p < GV_COLS / 2; ++p) acc2[p][m] = fma2(wp[p][j], xx, acc2[p][m]);
-                }
-            }
-        }
-    }
-    // sums over the lanes (every lane ends with all of them), then lane c * MR + m finishes element (m, n0 + c)
-    float mine = 0.f;
-#pragma unroll
-    for (int c = 0; c < GV_COLS; ++c)
-#pragma unroll
-        for (int m = 0; m < MR; ++m) {
-            float lo, hi;
-            unpack2(acc2[c >> 1][m], lo, hi);
-            float v = (c & 1) ? hi : lo;
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (lane == c * MR + m) mine = v;
-        }
-    float contrib = 0.f;
-    if (lane < GV_COLS * MR) {
-        const int c = lane / MR, m = lane - c * MR, n = n0 + c;
-        if (m < P.M) {
-            const float z = mine + (P.bias ? __bfloat162float(P.bias[n]) : 0.f);
-            const float y = __bfloat162float(P.X[(size_t)m * d + n]) + silu(z);
-            if (P.Y) P.Y[(size_t)m * d + n] = __float2bfloat16_rn(y);
-            if (P.w_out) contrib = y * __bfloat162float(P.w_out[n]);
-        }
-    }
-    if (P.partial) {                                   // last block: one partial dot per (row, CTA), in a fixed order
-#pragma unroll
-        for (int o = MR; o < GV_COLS * MR; o <<= 1) contrib += __shfl_xor_sync(0xffffffffu, contrib, o);
-        if (lane < MR) dots[warp][lane] = contrib;
-        __syncthreads();
-        const int nt = d / GV_TILE;
-        if (tid < MR && tid < P.M) {
-            float sum = 0.f;
-#pragma unroll
-            for (int w = 0; w < GV_WARPS; ++w) sum += dots[w][tid];
-            P.partial[(size_t)tid * nt + blockIdx.x] = sum;
-        }
-        // the last CTA to get here finishes the head: accept_prob[m] = sigmoid(sum_t partial[m, t] + b_out),
-        // a warp per row, added in a fixed order
-        __shared__ int last;
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) last = (atomicAdd(P.done_ctr, 1) == (int)gridDim.x - 1);
-        __syncthreads();
-        if (last) {
-            __threadfence();
-            if (warp < P.M) {
-                float v = 0.f;
-                for (int t = lane; t < nt; t += 32) v += __ldcg(P.partial + (size_t)warp * nt + t);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                if (lane == 0) P.accept_prob[warp] = 1.f / (1.f + __expf(-(v + P.b_out)));
-            }
-            if (tid == 0) *P.done_ctr = 0;             // ready for the next call
-        }
-    }
-}
-
-template <int MR>
-cudaError_t launch_rows(const BlockParams& p, cudaStream_t s) {
-    const size_t smem = (size_t)MR * p.d * 2;
-    if (smem > 40 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(head_rows_kernel<MR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-    }
-    head_rows_kernel<MR><<<p.d / GV_TILE, GV_THREADS, smem, s>>>(p);
-    return cudaGetLastError();
-}
-
-// ---------------------------------------------------------------------------------------------
-// The block for up to 16 rows on warp-level tensor-core instructions (mma.sync m16n8k16): still a
-// stream of the weights, but the multiply-adds no longer load the CUDA cores.  A CTA owns 32
-// output columns (four 8-column tiles); its 16 warps split k, so that every lane has 16 vectors of
-// weights in flight and the CTA 128 KB.  A lane's 16-byte vector holds eight consecutive k of one
-// column; since a dot product does not care about the order of k, those eight feed two MMAs with
-// the rows of X read from shared memory in the same order.  The warps' partial tiles are added
-// through shared memory in a fixed order; epilogue and finish as in the kernel above.
-constexpr int MM_WARPS = 16, MM_THREADS = MM_WARPS * 32, MM_TILE = 32, MM_NT = MM_TILE / 8, MM_ROWS = 16;
-constexpr int MM_PAD = 64;                             // bytes added to a row of X in shared memory (bank spread)
-
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-__global__ void __launch_bounds__(MM_THREADS, 1) head_mma16_kernel(const BlockParams P) {
-    extern __shared__ __align__(16) unsigned char mm_smem[];
-    const int d = P.d, row_bytes = d * 2 + MM_PAD;
-    unsigned char* xs = mm_smem;                                          // [16][row_bytes]: rows of X, bf16
-    float* red = reinterpret_cast<float*>(mm_smem + MM_ROWS * row_bytes); // [MM_WARPS][MM_NT][32][4]
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const int n0 = blockIdx.x * MM_TILE;
-    const int kslice = d / MM_WARPS, nchunk = kslice / 32, kbase = warp * kslice;   // chunks of 32 k per warp
-    constexpr int CH = 4;                                                 // chunks per round: 16 vectors in flight per lane
-
-    const uint4* wp[MM_NT];
-#pragma unroll
-    for (int j = 0; j < MM_NT; ++j)
-        wp[j] = reinterpret_cast<const uint4*>(P.W + (size_t)(n0 + j * 8 + g) * d + kbase + t * 8);
-    uint4 wv[CH][MM_NT];
-#pragma unroll
-    for (int u = 0; u < CH; ++u)
-#pragma unroll
-        for (int j = 0; j < MM_NT; ++j) wv[u][j] = u < nchunk ? __ldcs(wp[j] + u * 4) : make_uint4(0, 0, 0, 0);
-
-    // rows of X into shared memory while the first weights are in flight
-    const int dv = d >> 3;
-    for (int i = tid; i < MM_ROWS * dv; i += MM_THREADS) {
-        const int m = i / dv, v = i - m * dv;
-        const uint4 x = m < P.M ? __ldg(reinterpret_cast<const uint4*>(P.X) + (size_t)m * dv + v) : make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(xs + (size_t)m * row_bytes + v * 16) = x;
-    }
-    __syncthreads();
-
-    float acc[MM_NT][4];
-#pragma unroll
-    for (int j = 0; j < MM_NT; ++j)
-#pragma unroll
-        for (int q = 0; q < 4; ++q) acc[j][q] = 0.f;
-    for (int c0 = 0; c0 < nchunk; c0 += CH) {
-#pragma unroll
-        for (int u = 0; u < CH; ++u) {
-            if (c0 + u >= nchunk) break;
-            const int k = kbase + (c0 + u) * 32 + t * 8;                  // this lane's eight k
-            const uint4 xa = *reinterpret_cast<const uint4*>(xs + (size_t)g * row_bytes + k * 2);
-            const uint4 xb = *reinterpret_cast<const uint4*>(xs + (size_t)(g + 8) * row_bytes + k * 2);
-            const int nx = c0 + CH + u;                                   // the slot is refilled as soon as it is used
-#pragma unroll
-            for (int j = 0; j < MM_NT; ++j) {
-                mma_bf16_16816(acc[j], xa.x, xb.x, xa.y, xb.y, wv[u][j].x, wv[u][j].y);
-                mma_bf16_16816(acc[j], xa.z, xb.z, xa.w, xb.w, wv[u][j].z, wv[u][j].w);
-                if (nx < nchunk) wv[u][j] = __ldcs(wp[j] + nx * 4);
-            }
-        }
-    }
-    // partial tiles of the 16 warps -> shared memory -> one thread per output element, fixed order
-#pragma unroll
-    for (int j = 0; j < MM_NT; ++j)
-        *reinterpret_cast<float4*>(red + (((size_t)warp * MM_NT + j) * 32 + lane) * 4) =
-            make_float4(acc[j][0], acc[j][1], acc[j][2], acc[j][3]);
-    __syncthreads();
-    const int row = tid >> 5, col = tid & 31;                             // a warp per row of the 16 x 32 tile
-    const int j = col >> 3, src_lane = (row & 7) * 4 + ((col & 7) >> 1), src_reg = (row >> 3) * 2 + (col & 1);
-    float z = 0.f;
-#pragma unroll
-    for (int w = 0; w < MM_WARPS; ++w) z += red[(((size_t)w * MM_NT + j) * 32 + src_lane) * 4 + src_reg];
-    const int n = n0 + col;
-    float contrib = 0.f;
-    if (row < P.M) {
-        z += P.bias ? __bfloat162float(P.bias[n]) : 0.f;
-        const float x = __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(xs + (size_t)row * row_bytes + n * 2));
-        const float y = x + silu(z);
-        if (P.Y) P.Y[(size_t)row * d + n] = __float2bfloat16_rn(y);
-        if (P.w_out) contrib = y * __bfloat162float(P.w_out[n]);
-    }
-    if (P.partial) {                                   // last block: partial dot per (row, CTA), then the finish
-        const int nt = d / MM_TILE;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xffffffffu, contrib, o);
-        if (lane == 0 && row < P.M) P.partial[(size_t)row * nt + blockIdx.x] = contrib;
-        __shared__ int last;
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) last = (atomicAdd(P.done_ctr, 1) == (int)gridDim.x - 1);
-        __syncthreads();
-        if (last) {
-            __threadfence();
-            if (warp < P.M) {
-                float v = 0.f;
-                for (int q = lane; q < nt; q += 32) v += __ldcg(P.partial + (size_t)warp * nt + q);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                if (lane == 0) P.accept_prob[warp] = 1.f / (1.f + __expf(-(v + P.b_out)));
-            }
-            if (tid == 0) *P.done_ctr = 0;
-        }
-    }
-}
-
-cudaError_t launch_mma16(const BlockParams& p, cudaStream_t s) {
-    const size_t smem = (size_t)MM_ROWS * (p.d * 2 + MM_PAD) + (size_t)MM_WARPS * MM_NT * 32 * 4 * sizeof(float);
-    cudaError_t e = cudaFuncSetAttribute(head_mma16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    head_mma16_kernel<<<p.d / MM_TILE, MM_THREADS, smem, s>>>(p);
-    return cudaGetLastError();
-}
-
 // accept_prob[m] = sigmoid(sum_t partial[m, t] + b_out)
 __global__ void head_finish_kernel(const float* __restrict__ partial, int M, int nt, float b_out,
                                    float* __restrict__ accept_prob) {
@@ -993,13 +723,9 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
     // few rows (the online, one-token-per-call use): narrow column tiles so that the weight stream is
     // spread over many SMs; otherwise the widest tile the width allows
     const int BN = d % 256 == 0 ? 256 : 128;
-    // 17 to 256 rows: the weights as the M-side operand, N = the rows rounded up to 16
+    // up to 256 rows: the weights as the M-side operand, N = the rows rounded up to 16
     const int Npad = (int)((M + 15) / 16 * 16);
-    // a handful of rows: the weight stream on the CUDA cores (no tensor maps needed)
-    // 5 to 16 rows: the same stream through warp-level MMAs (X rows in shared memory: d <= 4096)
-    const bool mma16_path = M > 4 && M <= MM_ROWS && d % 512 == 0 && d <= 4096;
-    const bool rows_path = !mma16_path && M <= 8 && d % 256 == 0 && d <= 8192;
-    const bool swap_path = !mma16_path && !rows_path && M <= 256;
+    const bool swap_path = M <= 256;
     for (int k = 0; k < D; ++k) {
         const void* W = head->W[k];
         const void* bias = head->b ? head->b[k] : nullptr;
@@ -1007,8 +733,7 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
             return fail(ctx, SPECDEC_EINVAL, "accept_head: weights and biases must be non-null and 16-byte aligned");
         const bool last = (k == D - 1);
         CUtensorMap mx, mw;
-        if (!rows_path && !mma16_path && (!cached_map(ctx, &mx, x, (int)M, d, swap_path ? Npad : BM) ||
-                                          !cached_map(ctx, &mw, W, d, d, swap_path ? BM : BN)))
+        if (!cached_map(ctx, &mx, x, (int)M, d, swap_path ? Npad : BM) || !cached_map(ctx, &mw, W, d, d, swap_path ? BM : BN))
             return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
         BlockParams p;
         p.X = x;
@@ -1021,19 +746,16 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
         p.d = d;
         p.sm_count = ctx->sm_count;
         p.status = ctx->status;
-        p.done_ctr = ctx->task_ctl + (swap_path ? 6 : 5);
+        p.done_ctr = ctx->task_ctl + 6;
         p.accept_prob = accept_prob;
         p.b_out = head->b_out;
-        cudaError_t e = mma16_path ? launch_mma16(p, s)
-                        : rows_path ? (M <= 1 ? launch_rows<1>(p, s) : M <= 2 ? launch_rows<2>(p, s)
-                                     : M <= 4 ? launch_rows<4>(p, s) : launch_rows<8>(p, s))
-                        : swap_path ? launch_swap(mx, mw, p, Npad, s)
+        cudaError_t e = swap_path ? launch_swap(mx, mw, p, Npad, s)
                         : BN == 256 ? launch_block<256>(mx, mw, p, s) : launch_block<128>(mx, mw, p, s);
         if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
         ctx->launches += 1;
         x = p.Y;
     }
-    if (!rows_path && !mma16_path && !swap_path) {
+    if (!swap_path) {
         head_finish_kernel<<<(int)((M + 127) / 128), 128, 0, s>>>(ctx->head_partial, (int)M, 2 * d / BN, head->b_out, accept_prob);
         ctx->launches += 1;
     }

@@ -27,7 +27,7 @@ struct specdec_ctx {
     unsigned long long* early_exits = nullptr;   // logit rows not read by units that left early (SPECDEC_VERIFY_EARLY_EXIT) since last read
     float4* norms = nullptr;      // [max_B * (max_K+1)]  log2 normalisers {hi_p, lo_p, hi_q, lo_q} per position
     int2* tasks = nullptr;        // [max_B]              rows whose y' is still to be drawn: {b, n}
-    int32_t* task_ctl = nullptr;  // [8]                  two-launch path: {tasks, finished CTAs}; fused path: {-, -, -, head, finished}; [5], [6]: CTAs done in the last head block (few-row kernels, weights-as-M kernel)
+    int32_t* task_ctl = nullptr;  // [8]                  two-launch path: {tasks, finished CTAs}; fused path: {-, -, -, head, finished}; [6]: CTAs done in the last block of the weights-as-M head kernel
     int32_t* task_ready = nullptr;// [max_B]              fused path: record {epoch:24, mode:2, n:6} of each resolved row
     uint32_t epoch = 0;
     uint64_t launches = 0;

@@ -73,8 +73,9 @@ def test_head_many_row_tiles(rows, d, depth):
 @pytest.mark.parametrize("rows", [1, 2, 3, 4, 5, 8, 9, 13, 16, 17, 32, 33, 64, 65])
 @pytest.mark.parametrize("d,depth,with_bias", [(256, 1, True), (512, 3, False), (4096, 2, True)])
 def test_head_few_rows(rows, d, depth, with_bias):
-    """At most 8 rows (one drafted token for a few sequences) take the weight-streaming kernel; row counts
-    that are not powers of two leave zero-padded rows."""
+    """One drafted token for 1 to 65 sequences (the weights-as-M kernel): row counts that are not multiples of
+    16 leave zero-padded accumulator columns; d = 256 splits the reduction over 4 CTAs of 1 k-block each,
+    d = 4096 of 16."""
     ctx = specdec.Context(rows, 1, max_d=d)
     hidden, Ws, bs, w_out, b_out = _head_problem(700 + rows + d, rows, 1, d, depth, with_bias, std=0.02 if d > 512 else 0.05)
     got = _run_head(ctx, hidden, Ws, bs, w_out, b_out)
@@ -170,7 +171,7 @@ def test_head_up_to_256_rows_at_full_width(rows):
 
 
 def test_online_head_and_stop_step_replay_algorithm_1():
-    """Algorithm 1's loop, one drafted token per call: head on [B,1,d] (few-row / weights-as-M kernels), then
+    """Algorithm 1's loop, one drafted token per call: head on [B,1,d] (weights-as-M kernel), then
     specdec_stop_step.  Each step is checked against the oracle; the replay must also reproduce the
     batched head + stop rule."""
     B, K, d = 96, 6, 512
