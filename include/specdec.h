@@ -14,7 +14,8 @@
  *   - Every pointer marked "dev" is device memory of the context's GPU, owned by the
  *     caller, neither retained nor freed by the library.  "host" pointers are ordinary
  *     (preferably pinned) host memory.
- *   - Tensors are dense row-major with the last index fastest.
+ *   - Tensors are dense row-major with the last index fastest; logit tensors start on a 4-byte boundary
+ *     (16-byte boundaries and rows of whole 16-byte vectors take the vectorised paths).
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the
  *     legacy default stream) unless stated otherwise; outputs are valid once the
  *     stream has been synchronised.

@@ -38,6 +38,8 @@ int check_verify_args(specdec_ctx* ctx, const void* target, const void* draft, i
     if (!target || !draft || !tokens || !uniforms || !n_acc || !next)
         return fail(ctx, SPECDEC_EINVAL, "verify_correct: null pointer argument");
     if (dtype != SPECDEC_F32 && dtype != SPECDEC_BF16) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown dtype %d", dtype);
+    if (reinterpret_cast<uintptr_t>(target) % 4 != 0 || reinterpret_cast<uintptr_t>(draft) % 4 != 0)
+        return fail(ctx, SPECDEC_EINVAL, "verify_correct: logit tensors must be 4-byte aligned");
     if (B < 1 || K < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "verify_correct: B, K, V must be >= 1 (got %d, %d, %d)", B, K, V);
     if (!(T > 0.f) || !std::isfinite(T)) return fail(ctx, SPECDEC_EINVAL, "verify_correct: temperature must be positive and finite");
     if ((flags & ~SPECDEC_VERIFY_EARLY_EXIT) > SPECDEC_VERIFY_CLUSTER) return fail(ctx, SPECDEC_EINVAL, "verify_correct: unknown flags %u", flags);
@@ -295,6 +297,7 @@ int specdec_sample(specdec_ctx* ctx, const void* logits, specdec_dtype dtype, co
     if (!logits || !uniforms || !tokens) return fail(ctx, SPECDEC_EINVAL, "sample: null pointer argument");
     if ((int)dtype != SPECDEC_F32 && (int)dtype != SPECDEC_BF16) return fail(ctx, SPECDEC_EINVAL, "sample: unknown dtype %d", (int)dtype);
     if (!(temperature > 0.f) || !std::isfinite(temperature)) return fail(ctx, SPECDEC_EINVAL, "sample: temperature must be positive and finite");
+    if (reinterpret_cast<uintptr_t>(logits) % 4 != 0) return fail(ctx, SPECDEC_EINVAL, "sample: logits must be 4-byte aligned");
     if (V > (1 << 22)) return fail(ctx, SPECDEC_EUNSUPPORTED, "sample: V=%d above 2^22", V);
     if (B < 1 || V < 1) return fail(ctx, SPECDEC_EINVAL, "sample: B and V must be >= 1 (got %d, %d)", B, V);
     if (B > ctx->max_B) return fail(ctx, SPECDEC_EUNSUPPORTED, "sample: B=%d exceeds the context (max_B=%d)", B, ctx->max_B);

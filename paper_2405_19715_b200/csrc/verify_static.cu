@@ -76,6 +76,8 @@ extern "C" int specdec_verify_correct_static(const void* target_logits, const vo
         return report(err, err_len, SPECDEC_EINVAL, "verify_correct_static: null pointer argument");
     if (dtype != SPECDEC_F32 && dtype != SPECDEC_BF16)
         return report(err, err_len, SPECDEC_EINVAL, "verify_correct_static: unknown dtype %d", (int)dtype);
+    if (reinterpret_cast<uintptr_t>(target_logits) % 4 != 0 || reinterpret_cast<uintptr_t>(draft_logits) % 4 != 0)
+        return report(err, err_len, SPECDEC_EINVAL, "verify_correct_static: logit tensors must be 4-byte aligned");
     if (B < 1 || K < 1 || V < 1)
         return report(err, err_len, SPECDEC_EINVAL, "verify_correct_static: B, K, V must be >= 1");
     if (!(temperature > 0.f) || temperature > 3.0e38f)
