@@ -725,7 +725,7 @@ def run_head_phases(args):
     out = torch.empty(M, 1, dtype=torch.float32, device="cuda")
     if M > 256:                                     # the 128-row-tile kernel: per-tile stamps of its first and last CTA
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        tl, ms = [], []
+        tl, ms, cy = [], [], []
         for i in range(max(args.steps, 3) + 3):
             torch.cuda.synchronize()
             e0.record()
@@ -734,20 +734,27 @@ def run_head_phases(args):
             torch.cuda.synchronize()
             buf = (ctypes.c_longlong * 128)()
             lib.specdec_debug_head_tile_stamps(buf)
-            a = np.array(buf[:], dtype=np.float64).reshape(2, 8, 8)[:, :, :6]
+            raw = np.array(buf[:], dtype=np.float64).reshape(2, 8, 8)
+            a = raw[:, :, :6]
             if i >= 3:
                 tl.append(np.where(a > 0, (a - a[a > 0].min()) * 1e-3, np.nan))
+                cy.append(np.where(raw[:, :, 3] > 0, raw[:, :, 7] - raw[:, :, 6], np.nan))   # main loop, SM cycles
                 ms.append(e0.elapsed_time(e1))
-        a = np.nanmedian(np.stack(tl), 0)
+        import warnings
+        with warnings.catch_warnings():              # tiles a CTA does not have are NaN in every call
+            warnings.simplefilter("ignore", RuntimeWarning)
+            a = np.nanmedian(np.stack(tl), 0)
+            cyc = np.nanmedian(np.stack(cy), 0)
         print(f"acceptance head, M={M} rows, d={d}, D={D}: tiles of the LAST block's launch on its first CTA (4 tiles at M=4096) and its "
               f"last CTA (3 tiles); microseconds from that launch's first stamp, median of {len(tl)} isolated calls; "
               f"whole call by CUDA events {1e3 * np.mean(ms):.1f} us")
-        print("| CTA | tile | first k-block requested | accumulator free | first k-block landed | all MMAs issued | accumulator complete | epilogue done |\n|---|---|---|---|---|---|---|---|")
+        print("| CTA | tile | first k-block requested | accumulator free | first k-block landed | all MMAs issued | accumulator complete | epilogue done | main loop (landed to issued), SM cycles | SM MHz in it |\n|---|---|---|---|---|---|---|---|---|---|")
         f = lambda v: "-" if np.isnan(v) else f"{v:.2f}"
         for c in range(2):
             for t in range(8):
                 if not np.isnan(a[c, t, 3]):
-                    print(f"| {'first' if c == 0 else 'last'} | {t} | " + " | ".join(f(a[c, t, k]) for k in range(6)) + " |")
+                    print(f"| {'first' if c == 0 else 'last'} | {t} | " + " | ".join(f(a[c, t, k]) for k in range(6))
+                          + f" | {cyc[c, t]:.0f} | {cyc[c, t] / (a[c, t, 3] - a[c, t, 2]):.0f} |")
         ctx.close()
         return
     rows = []

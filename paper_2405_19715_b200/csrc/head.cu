@@ -55,15 +55,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: on exhaustion a status bit is set and execution simply continues, so every
-// thread still reaches the barriers and the tensor-memory release below.
-// `budget` is the calling thread's poll allowance: after one give-up the later waits of that thread
-// are short, so a broken pipeline drains in about a second instead of one limit per wait.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, uint32_t* status, uint32_t& budget) {
-    for (uint32_t it = 0; it < budget; ++it)
-        if (mbar_try_wait(bar, parity)) return;
-    atomicOr(status, SPECDEC_DATA_WAIT_LIMIT);
-    budget = 1024;
+// Bounded wait: when the polls run out the thread simply continues, so it still reaches the barriers and
+// the tensor-memory release below; `budget` is the calling thread's poll allowance, cut to WAIT_POLLS_LEFT by
+// a give-up, so that a broken pipeline drains in about a second instead of one limit per wait, and
+// report_wait_limit() at the end of the kernel turns a cut allowance into the status bit.
+// The wait is only a probe loop on registers: in the MMA-issuing thread the barrier has nearly always
+// completed already, and with the status update inside the wait that thread needed ~100 cycles more per
+// k-block than the tensor pipe does (measured: 643 against 547 cycles per k-block, 512 being the pipe's).
+constexpr uint32_t WAIT_POLLS_LEFT = 1024;
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, uint32_t& budget) {
+    for (uint32_t n = 0; !mbar_try_wait(bar, parity); ++n)
+        if (n >= budget) {
+            budget = WAIT_POLLS_LEFT;
+            return;
+        }
+}
+__device__ __forceinline__ void report_wait_limit(uint32_t* status, uint32_t budget) {
+    if (budget != WAIT_POLLS) atomicOr(status, SPECDEC_DATA_WAIT_LIMIT);
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
@@ -86,6 +94,31 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// The four MMAs of one 64-wide k-block in one statement.  `a_lo`, `b_lo` are the low words of the operands'
+// descriptors at k = 0 (address >> 4 in bits 0-13, leading offset in bit 16); a step of 16 bf16 along K is 32
+// bytes, i.e. + 2 in that word, and the high word (stride, version, swizzle) is the same for every tile, so
+// the issuing thread spends one add per descriptor instead of rebuilding 64-bit values.  `acc_first` is the
+// accumulate flag of the first MMA (0 on a tile's first k-block); the other three always accumulate.
+constexpr uint32_t UMMA_DESC_HI = 64u | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr) { return ((smem_addr >> 4) & 0x3FFFu) | (1u << 16); }
+__device__ __forceinline__ void umma_kblock(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t.reg .b32 ta, tb;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.eq.b32 q, 0, 0;\n\t"
+        "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t"
+        "add.u32 ta, %1, 2;\n\tadd.u32 tb, %2, 2;\n\t"
+        "mov.b64 da, {ta, %5};\n\tmov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, q;\n\t"
+        "add.u32 ta, %1, 4;\n\tadd.u32 tb, %2, 4;\n\t"
+        "mov.b64 da, {ta, %5};\n\tmov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, q;\n\t"
+        "add.u32 ta, %1, 6;\n\tadd.u32 tb, %2, 6;\n\t"
+        "mov.b64 da, {ta, %5};\n\tmov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, q;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(acc_first), "r"(UMMA_DESC_HI) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -128,7 +161,8 @@ struct BlockParams {
 
 // Per-tile timestamps of the first and the last CTA (diagnostic builds only): [CTA 0 / last][tile][slot], ns of
 // the global timer.  Slots: 0 TMA warp requests the tile's first k-block, 1 MMA warp has a free accumulator,
-// 2 first k-block landed, 3 all MMAs issued, 4 epilogue sees the accumulator complete, 5 epilogue done.
+// 2 first k-block landed, 3 all MMAs issued, 4 epilogue sees the accumulator complete, 5 epilogue done;
+// 6 and 7 hold the SM's cycle counter at stamps 2 and 3 (cycles of the main loop, and with the timer its clock).
 #ifdef SPECDEC_STAMPS
 __device__ long long head_tile_stamps[2 * 8 * 8];
 #define TILE_STAMP(it, slot)                                                                          \
@@ -137,6 +171,8 @@ __device__ long long head_tile_stamps[2 * 8 * 8];
             long long t_;                                                                             \
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                    \
             head_tile_stamps[((blockIdx.x == 0 ? 0 : 1) * 8 + (it)) * 8 + (slot)] = t_;               \
+            if ((slot) == 2 || (slot) == 3)                                                           \
+                head_tile_stamps[((blockIdx.x == 0 ? 0 : 1) * 8 + (it)) * 8 + (slot) + 4] = clock64(); \
         }                                                                                             \
     } while (0)
 #else
@@ -193,7 +229,7 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
                 const int m0 = (t / ntn) * BM, n0 = (t % ntn) * BN;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    mbar_wait(empty0 + 8 * stage, phase ^ 1u, P.status, budget);
+                    mbar_wait(empty0 + 8 * stage, phase ^ 1u, budget);
                     if (kb == 0) TILE_STAMP(it, 0);
                     const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
                     mbar_expect_tx(full0 + 8 * stage, C::STAGE_BYTES);
@@ -207,22 +243,21 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = umma_idesc(BN);
+            static_assert(BK / UMMA_K == 4, "umma_kblock issues four MMAs");
+            const uint32_t desc_lo0 = umma_desc_lo(base);      // stage 0 of the ring, operand A, k = 0
             uint32_t stage = 0, phase = 0, it = 0;
             for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
                 const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
-                mbar_wait(tempty0 + 8 * buf, use ^ 1u, P.status, budget);      // epilogue has drained this accumulator
+                mbar_wait(tempty0 + 8 * buf, use ^ 1u, budget);      // epilogue has drained this accumulator
                 TILE_STAMP(it, 1);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t acc = tmem + buf * BN;
                 for (int kb = 0; kb < nkb; ++kb) {
-                    mbar_wait(full0 + 8 * stage, phase, P.status, budget);
+                    mbar_wait(full0 + 8 * stage, phase, budget);
                     if (kb == 0) TILE_STAMP(it, 2);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k)
-                        umma_bf16(acc, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), idesc,
-                                  (kb | k) != 0 ? 1u : 0u);
+                    const uint32_t a_lo = desc_lo0 + stage * (C::STAGE_BYTES >> 4);
+                    umma_kblock(acc, a_lo, a_lo + (C::A_BYTES >> 4), idesc, kb != 0 ? 1u : 0u);
                     umma_commit(empty0 + 8 * stage);          // stage reusable once these MMAs have read it
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -245,7 +280,7 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             uint4 xv[4], xn[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) xn[j] = row_ok ? __ldg(xrow + (half * CH) * 4 + j) : make_uint4(0, 0, 0, 0);
-            mbar_wait(tfull0 + 8 * buf, use, P.status, budget);
+            mbar_wait(tfull0 + 8 * buf, use, budget);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (warp == 2 && lane == 0) TILE_STAMP(it, 4);
             float dot = 0.f;
@@ -289,6 +324,7 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             if (P.partial && row_ok) P.partial[(size_t)m * (2 * ntn) + 2 * (t % ntn) + half] = dot;
         }
     }
+    report_wait_limit(P.status, budget);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
@@ -405,7 +441,7 @@ head_swap_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
                 tma_load_2d(base + kb * stage_bytes + a_bytes, &mapX, (kb0 + kb) * BK, 0, full0 + 8 * kb);
             uint32_t stage = 0, phase = 1;                                // the ring has been filled once
             for (int kb = ahead; kb < nkb; ++kb) {
-                mbar_wait(empty0 + 8 * stage, phase ^ 1u, P.status, budget);
+                mbar_wait(empty0 + 8 * stage, phase ^ 1u, budget);
                 const uint32_t a = base + stage * stage_bytes, b = a + a_bytes;
                 mbar_expect_tx(full0 + 8 * stage, stage_bytes);
                 tma_load_2d(a, &mapW, (kb0 + kb) * BK, n0, full0 + 8 * stage);     // 128 weight rows
@@ -418,7 +454,7 @@ head_swap_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
             const uint32_t idesc = umma_idesc(Npad);
             uint32_t stage = 0, phase = 0;
             for (int kb = 0; kb < nkb; ++kb) {
-                mbar_wait(full0 + 8 * stage, phase, P.status, budget);
+                mbar_wait(full0 + 8 * stage, phase, budget);
                 if (kb == 0) HEAD_STAMP(2);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t a = base + stage * stage_bytes, b = a + a_bytes;
@@ -440,7 +476,7 @@ head_swap_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
             const int m = (warp - 2) + 4 * u;
             xr[u] = m < P.M ? __ldg(xcol + (size_t)m * P.d) : (unsigned short)0;
         }
-        mbar_wait(tfull, 0, P.status, budget);                            // this CTA's accumulator is complete
+        mbar_wait(tfull, 0, budget);                            // this CTA's accumulator is complete
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         HEAD_STAMP(4);
     }
@@ -540,6 +576,7 @@ head_swap_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
             if (tid == 0) *P.done_ctr = 0;                                // ready for the next call
         }
     }
+    report_wait_limit(P.status, budget);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     HEAD_STAMP(9);
