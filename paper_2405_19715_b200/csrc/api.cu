@@ -96,6 +96,8 @@ int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_
         if (e == cudaSuccess) e = cudaMalloc(&ctx->act[1], act);
         if (e == cudaSuccess)
             e = cudaMalloc(&ctx->head_partial, (size_t)max_B * max_K * ((max_d + 31) / 32) * sizeof(float));
+        if (e == cudaSuccess)
+            e = cudaMalloc(&ctx->head_ready, 8 * (((size_t)max_B * max_K + 127) / 128) * sizeof(uint32_t));
     }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -123,6 +125,7 @@ int specdec_destroy(specdec_ctx* ctx) {
     cudaFree(ctx->act[0]);
     cudaFree(ctx->act[1]);
     cudaFree(ctx->head_partial);
+    cudaFree(ctx->head_ready);
     delete ctx;
     return SPECDEC_OK;
 }

@@ -5,9 +5,9 @@
 // are K-major) on the 5th-generation tensor cores: operand tiles arrive in shared memory by TMA
 // (128-byte swizzle), one thread issues tcgen05.mma with the fp32 accumulator in tensor memory,
 // and eight epilogue warps read the (double-buffered) accumulator back with tcgen05.ld and apply
-// bias, SiLU and the residual while the next tile's MMAs run.  The last block does not store x_D: its epilogue multiplies by w_out and leaves
-// one partial dot product per (row, column tile); a small kernel adds them and applies the
-// sigmoid.  D = 0 is a plain row-times-vector kernel.
+// bias, SiLU and the residual while the next tile's MMAs run.  The last block does not store x_D: its
+// epilogue multiplies by w_out and leaves one partial dot product per (row, column tile); whoever
+// finishes a row's last tile adds them and applies the sigmoid.  D = 0 is a plain row-times-vector kernel.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -179,13 +179,47 @@ __device__ long long head_tile_stamps[2 * 8 * 8];
 #define TILE_STAMP(it, slot) do {} while (0)
 #endif
 
-// Persistent: CTA c works on tiles c, c + grid, ... (column tile fastest).  The accumulator is
-// double-buffered in tensor memory (2 x BN columns), so the epilogue of one tile runs while the
-// MMAs of the next are issued.
+// The residual blocks of one call as ONE launch (more than 256 rows).
+constexpr int CHAIN_MAX = 8;                       // residual blocks per launch (the entry point's depth limit)
+constexpr uint32_t FLAG_POLLS = 1u << 21;          // polls of a row block's counter before giving up (~ a second)
+struct ChainLayer {
+    const __nv_bfloat16* X;      // [M, d] input of the block (also the residual)
+    const __nv_bfloat16* bias;   // [d] or null
+    __nv_bfloat16* Y;            // [M, d] output; null for the block that ends the head
+};
+struct ChainParams {
+    CUtensorMap mapX[CHAIN_MAX], mapW[CHAIN_MAX];
+    ChainLayer layer[CHAIN_MAX];
+    int first, end;              // blocks [first, end) are computed by this launch
+    int depth;                   // blocks of the head: block depth - 1 multiplies by w_out instead of storing
+    int M, d;
+    const __nv_bfloat16* w_out;  // [d]
+    float* partial;              // [M, 2 * d / BN] partial dots of the last block
+    uint32_t* ready;             // [depth][row blocks] epilogue warps that have finished a tile of (block, row block)
+    float* accept_prob;
+    float b_out;
+    uint32_t* status;
+};
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Persistent over the tiles of all its blocks: tile g = (block, row block, column tile), column tile fastest,
+// block slowest; CTA c works on tiles c, c + grid, ...  A tile of block l > first reads rows that the 128-row
+// tiles of block l - 1 in the same row block wrote, so its TMA thread first waits until `ready` shows all of
+// them finished (every epilogue warp counts once per tile, after its stores).  Those tiles come earlier in the
+// order, so with all CTAs resident (the launch is cooperative) the tile with the lowest unfinished index never
+// waits for an unfinished one; the wait is bounded all the same.  With 512 tiles per block on 148 SMs two blocks
+// take 7 rounds in one launch instead of 4 + 4 in two, and only the first tile of the launch waits for its
+// operands with nothing to overlap.  The accumulator is double-buffered in tensor memory (2 x BN columns), so
+// the epilogue of one tile runs while the MMAs of the next are issued.  In the head's last block the warp that
+// completes a row block's count adds the block's partial dots in column order and applies the sigmoid.
 template <int BN>
 __global__ void __launch_bounds__(HEAD_THREADS, 1)
-head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
-                  const BlockParams P) {
+head_chain_kernel(const __grid_constant__ ChainParams P) {
     using C = Cfg<BN>;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
@@ -197,7 +231,9 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int nkb = P.d / BK;
-    const int ntn = P.d / BN, ntiles = ntn * ((P.M + BM - 1) / BM);
+    const int ntn = P.d / BN, ntm = (P.M + BM - 1) / BM, per_block = ntn * ntm;
+    const int ntiles = (P.end - P.first) * per_block;
+    const uint32_t tile_warps = (uint32_t)(ntn * EPI_WARPS);              // counts that complete a row block
     uint32_t budget = WAIT_POLLS;
 
     if (tid == 0) {
@@ -226,15 +262,28 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, it = 0;
-            for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
+            for (int g = blockIdx.x; g < ntiles; g += gridDim.x, ++it) {
+                const int l = P.first + g / per_block, t = g % per_block;
                 const int m0 = (t / ntn) * BM, n0 = (t % ntn) * BN;
+                if (l > P.first) {                             // the rows of X come from this launch's previous block
+                    const uint32_t* ctr = P.ready + (size_t)(l - 1) * ntm + t / ntn;
+                    uint32_t polls = 0;
+                    while (ld_acquire_u32(ctr) < tile_warps)
+                        if (++polls >= (budget == WAIT_POLLS ? FLAG_POLLS : WAIT_POLLS_LEFT)) {
+                            budget = WAIT_POLLS_LEFT;
+                            break;
+                        }
+                    asm volatile("fence.proxy.async;" ::: "memory");   // the loads below go through the async proxy
+                }
+                const CUtensorMap* mx = &P.mapX[l];
+                const CUtensorMap* mw = &P.mapW[l];
                 for (int kb = 0; kb < nkb; ++kb) {
                     mbar_wait(empty0 + 8 * stage, phase ^ 1u, budget);
                     if (kb == 0) TILE_STAMP(it, 0);
                     const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
                     mbar_expect_tx(full0 + 8 * stage, C::STAGE_BYTES);
-                    tma_load_2d(a, &mapX, kb * BK, m0, full0 + 8 * stage);
-                    tma_load_2d(b, &mapW, kb * BK, n0, full0 + 8 * stage);
+                    tma_load_2d(a, mx, kb * BK, m0, full0 + 8 * stage);
+                    tma_load_2d(b, mw, kb * BK, n0, full0 + 8 * stage);
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -246,7 +295,7 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             static_assert(BK / UMMA_K == 4, "umma_kblock issues four MMAs");
             const uint32_t desc_lo0 = umma_desc_lo(base);      // stage 0 of the ring, operand A, k = 0
             uint32_t stage = 0, phase = 0, it = 0;
-            for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
+            for (int g = blockIdx.x; g < ntiles; g += gridDim.x, ++it) {
                 const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
                 mbar_wait(tempty0 + 8 * buf, use ^ 1u, budget);      // epilogue has drained this accumulator
                 TILE_STAMP(it, 1);
@@ -271,18 +320,24 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         const int half = (warp - 2) >> 2;                  // which half of the tile's columns
         constexpr int CH = BN / 32 / 2;                    // 32-column chunks per warp
         uint32_t it = 0;
-        for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
+        for (int g = blockIdx.x; g < ntiles; g += gridDim.x, ++it) {
+            const int l = P.first + g / per_block, t = g % per_block;
             const int m0 = (t / ntn) * BM, n0 = (t % ntn) * BN;
+            const bool last = l == P.depth - 1;
+            const __nv_bfloat16* bias = P.layer[l].bias;
+            const __nv_bfloat16* w_out = last ? P.w_out : nullptr;
+            __nv_bfloat16* Y = P.layer[l].Y;
             const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
             const int m = m0 + q * 32 + lane;
             const bool row_ok = m < P.M;
-            const uint4* xrow = reinterpret_cast<const uint4*>(P.X + (size_t)(row_ok ? m : 0) * P.d + n0);
+            // the residual may have been written by another SM during this launch: read it past L1
+            const uint4* xrow = reinterpret_cast<const uint4*>(P.layer[l].X + (size_t)(row_ok ? m : 0) * P.d + n0);
             uint4 xv[4], xn[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) xn[j] = row_ok ? __ldg(xrow + (half * CH) * 4 + j) : make_uint4(0, 0, 0, 0);
             mbar_wait(tfull0 + 8 * buf, use, budget);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (warp == 2 && lane == 0) TILE_STAMP(it, 4);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) xn[j] = row_ok ? __ldcg(xrow + (half * CH) * 4 + j) : make_uint4(0, 0, 0, 0);
             float dot = 0.f;
 #pragma unroll 1
             for (int cc = 0; cc < CH; ++cc) {
@@ -293,9 +348,9 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     xv[j] = xn[j];
-                    if (cc + 1 < CH) xn[j] = row_ok ? __ldg(xrow + (c + 1) * 4 + j) : make_uint4(0, 0, 0, 0);
-                    bv[j] = P.bias ? __ldg(reinterpret_cast<const uint4*>(P.bias + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
-                    wv[j] = P.w_out ? __ldg(reinterpret_cast<const uint4*>(P.w_out + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
+                    if (cc + 1 < CH) xn[j] = row_ok ? __ldcg(xrow + (c + 1) * 4 + j) : make_uint4(0, 0, 0, 0);
+                    bv[j] = bias ? __ldg(reinterpret_cast<const uint4*>(bias + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
+                    wv[j] = w_out ? __ldg(reinterpret_cast<const uint4*>(w_out + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
                 }
                 const uint32_t* xw = reinterpret_cast<const uint32_t*>(xv);
                 const uint32_t* bw = reinterpret_cast<const uint32_t*>(bv);
@@ -310,8 +365,8 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     const __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
                     out[j] = *reinterpret_cast<const uint32_t*>(&pk);
                 }
-                if (P.Y && row_ok) {
-                    uint4* yrow = reinterpret_cast<uint4*>(P.Y + (size_t)m * P.d + n0 + c * 32);
+                if (Y && row_ok) {
+                    uint4* yrow = reinterpret_cast<uint4*>(Y + (size_t)m * P.d + n0 + c * 32);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) yrow[j] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
                 }
@@ -321,7 +376,28 @@ head_block_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty0 + 8 * buf);
             if (warp == 2 && lane == 0) TILE_STAMP(it, 5);
-            if (P.partial && row_ok) P.partial[(size_t)m * (2 * ntn) + 2 * (t % ntn) + half] = dot;
+            if (last && row_ok) P.partial[(size_t)m * (2 * ntn) + 2 * (t % ntn) + half] = dot;
+            // count this warp's part of the tile as written; the count of a row block is what the next block's
+            // tiles (their TMA loads: the async proxy) and, in the last block, the row block's finisher wait for
+            __syncwarp();
+            uint32_t* ctr = P.ready + (size_t)l * ntm + t / ntn;
+            uint32_t before = 0;
+            if (lane == 0) {
+                __threadfence();                               // the warp's stores (ordered before by the barrier), then the count
+                before = atomicAdd(ctr, 1u);
+            }
+            before = __shfl_sync(0xffffffffu, before, 0);
+            if (last && before == tile_warps - 1) {            // every dot of this row block is in place
+                __threadfence();
+                for (int r = lane; r < BM; r += 32) {
+                    const int mr = m0 + r;
+                    if (mr >= P.M) break;
+                    const float* pr = P.partial + (size_t)mr * (2 * ntn);
+                    float sum = P.b_out;
+                    for (int c = 0; c < 2 * ntn; ++c) sum += __ldcg(pr + c);
+                    P.accept_prob[mr] = 1.f / (1.f + __expf(-sum));
+                }
+            }
         }
     }
     report_wait_limit(P.status, budget);
@@ -586,16 +662,6 @@ head_swap_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
     }
 }
 
-// accept_prob[m] = sigmoid(sum_t partial[m, t] + b_out)
-__global__ void head_finish_kernel(const float* __restrict__ partial, int M, int nt, float b_out,
-                                   float* __restrict__ accept_prob) {
-    const int m = blockIdx.x * blockDim.x + threadIdx.x;
-    if (m >= M) return;
-    float s = b_out;
-    for (int t = 0; t < nt; ++t) s += partial[(size_t)m * nt + t];
-    accept_prob[m] = 1.f / (1.f + __expf(-s));
-}
-
 // D = 0: one warp per row, accept_prob[m] = sigmoid(hidden[m, :] . w_out + b_out)
 __global__ void head_linear_kernel(const __nv_bfloat16* __restrict__ X, const __nv_bfloat16* __restrict__ w, int M,
                                    int d, float b_out, float* __restrict__ accept_prob) {
@@ -704,13 +770,32 @@ cudaError_t launch_swap(const CUtensorMap& mx, const CUtensorMap& mw, const Bloc
     return cudaLaunchKernelEx(&cfg, kern, mx, mw, p, Npad, stages, tmem_cols);
 }
 
+// Blocks [first, end) of the chain in one launch; cooperative when it spans more than one block (its CTAs
+// then wait for one another's tiles and must all be resident).
 template <int BN>
-cudaError_t launch_block(const CUtensorMap& mx, const CUtensorMap& mw, const BlockParams& p, cudaStream_t s) {
-    cudaError_t e = cudaFuncSetAttribute(head_block_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM);
-    if (e != cudaSuccess) return e;
-    const int ntiles = (p.d / BN) * ((p.M + BM - 1) / BM);
-    head_block_kernel<BN><<<ntiles < p.sm_count ? ntiles : p.sm_count, HEAD_THREADS, Cfg<BN>::SMEM, s>>>(mx, mw, p);
-    return cudaGetLastError();
+cudaError_t launch_chain(ChainParams& p, int first, int end, int sm_count, bool cooperative, cudaStream_t s) {
+    static unsigned long long allowed = 0;                                // per device: large dynamic shared memory granted
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!((allowed >> (dev & 63)) & 1ull)) {
+        cudaError_t e = cudaFuncSetAttribute(head_chain_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM);
+        if (e != cudaSuccess) return e;
+        allowed |= 1ull << (dev & 63);
+    }
+    p.first = first;
+    p.end = end;
+    const int ntiles = (end - first) * (p.d / BN) * ((p.M + BM - 1) / BM);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)std::min(ntiles, sm_count));             // one CTA per SM (its ring fills the shared memory)
+    cfg.blockDim = dim3(HEAD_THREADS);
+    cfg.dynamicSmemBytes = (size_t)Cfg<BN>::SMEM;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = cooperative ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, head_chain_kernel<BN>, p);
 }
 
 int fail(specdec_ctx* ctx, int code, const char* msg) {
@@ -768,33 +853,82 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
         const void* bias = head->b ? head->b[k] : nullptr;
         if (!W || reinterpret_cast<uintptr_t>(W) % 16 != 0 || (bias && reinterpret_cast<uintptr_t>(bias) % 16 != 0))
             return fail(ctx, SPECDEC_EINVAL, "accept_head: weights and biases must be non-null and 16-byte aligned");
-        const bool last = (k == D - 1);
-        CUtensorMap mx, mw;
-        if (!cached_map(ctx, &mx, x, (int)M, d, swap_path ? Npad : BM) || !cached_map(ctx, &mw, W, d, d, swap_path ? BM : BN))
-            return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
-        BlockParams p;
-        p.X = x;
-        p.W = static_cast<const __nv_bfloat16*>(W);
-        p.bias = static_cast<const __nv_bfloat16*>(bias);
-        p.Y = last ? nullptr : static_cast<__nv_bfloat16*>(ctx->act[k & 1]);
-        p.w_out = last ? static_cast<const __nv_bfloat16*>(head->w_out) : nullptr;
-        p.partial = last ? ctx->head_partial : nullptr;
+    }
+    if (swap_path) {
+        for (int k = 0; k < D; ++k) {
+            const bool last = (k == D - 1);
+            CUtensorMap mx, mw;
+            if (!cached_map(ctx, &mx, x, (int)M, d, Npad) || !cached_map(ctx, &mw, head->W[k], d, d, BM))
+                return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
+            BlockParams p;
+            p.X = x;
+            p.W = static_cast<const __nv_bfloat16*>(head->W[k]);
+            p.bias = static_cast<const __nv_bfloat16*>(head->b ? head->b[k] : nullptr);
+            p.Y = last ? nullptr : static_cast<__nv_bfloat16*>(ctx->act[k & 1]);
+            p.w_out = last ? static_cast<const __nv_bfloat16*>(head->w_out) : nullptr;
+            p.partial = last ? ctx->head_partial : nullptr;
+            p.M = (int)M;
+            p.d = d;
+            p.sm_count = ctx->sm_count;
+            p.status = ctx->status;
+            p.done_ctr = ctx->task_ctl + 6;
+            p.accept_prob = accept_prob;
+            p.b_out = head->b_out;
+            cudaError_t e = launch_swap(mx, mw, p, Npad, s);
+            if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
+            ctx->launches += 1;
+            x = p.Y;
+        }
+    } else {
+        ChainParams p;
+        for (int k = 0; k < D; ++k) {
+            if (!cached_map(ctx, &p.mapX[k], x, (int)M, d, BM) || !cached_map(ctx, &p.mapW[k], head->W[k], d, d, BN))
+                return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
+            p.layer[k].X = x;
+            p.layer[k].bias = static_cast<const __nv_bfloat16*>(head->b ? head->b[k] : nullptr);
+            p.layer[k].Y = k == D - 1 ? nullptr : static_cast<__nv_bfloat16*>(ctx->act[k & 1]);
+            x = p.layer[k].Y;
+        }
+        for (int k = D; k < CHAIN_MAX; ++k) {                  // unused slots: defined bytes for the parameter copy
+            p.mapX[k] = p.mapX[0];
+            p.mapW[k] = p.mapW[0];
+            p.layer[k] = ChainLayer{nullptr, nullptr, nullptr};
+        }
+        p.depth = D;
         p.M = (int)M;
         p.d = d;
-        p.sm_count = ctx->sm_count;
-        p.status = ctx->status;
-        p.done_ctr = ctx->task_ctl + 6;
+        p.w_out = static_cast<const __nv_bfloat16*>(head->w_out);
+        p.partial = ctx->head_partial;
+        p.ready = ctx->head_ready;
         p.accept_prob = accept_prob;
         p.b_out = head->b_out;
-        cudaError_t e = swap_path ? launch_swap(mx, mw, p, Npad, s)
-                        : BN == 256 ? launch_block<256>(mx, mw, p, s) : launch_block<128>(mx, mw, p, s);
+        p.status = ctx->status;
+        const size_t ntm = (size_t)((M + BM - 1) / BM);
+        cudaError_t e = cudaMemsetAsync(ctx->head_ready, 0, (size_t)D * ntm * sizeof(uint32_t), s);
         if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
-        ctx->launches += 1;
-        x = p.Y;
-    }
-    if (!swap_path) {
-        head_finish_kernel<<<(int)((M + 127) / 128), 128, 0, s>>>(ctx->head_partial, (int)M, 2 * d / BN, head->b_out, accept_prob);
-        ctx->launches += 1;
+        auto launch = [&](int first, int end, bool coop) {
+            return BN == 256 ? launch_chain<256>(p, first, end, ctx->sm_count, coop, s)
+                             : launch_chain<128>(p, first, end, ctx->sm_count, coop, s);
+        };
+        if (ctx->head_coop != 0 && D > 1) {
+            e = launch(0, D, true);
+            if (e == cudaSuccess) {
+                ctx->head_coop = 1;
+                ctx->launches += 1;
+            } else if (ctx->head_coop < 0 && (e == cudaErrorCooperativeLaunchTooLarge || e == cudaErrorNotSupported)) {
+                (void)cudaGetLastError();                          // this device or partition cannot hold the grid: one launch per block
+                ctx->head_coop = 0;
+            } else {
+                return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
+            }
+        }
+        if (ctx->head_coop == 0 || D == 1) {
+            for (int k = 0; k < D; ++k) {
+                e = launch(k, k + 1, false);
+                if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
+                ctx->launches += 1;
+            }
+        }
     }
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? SPECDEC_OK : fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
