@@ -27,13 +27,16 @@ constexpr int UMMA_K = 16;
 constexpr int EPI_WARPS = 8;             // two per 32-lane quarter of tensor memory, each taking half the columns
 constexpr int HEAD_THREADS = (2 + EPI_WARPS) * 32;   // warp 0 TMA, warp 1 MMA + tensor-memory owner, then epilogue
 constexpr uint32_t WAIT_POLLS = 1u << 24;
+constexpr int OUT_COLS = 32, OUT_ROWS = 32;                       // box of one TMA store of the output: 32 rows x 64 bytes
+constexpr int OUT_BOX_BYTES = OUT_ROWS * OUT_COLS * 2;
 
 template <int BN> struct Cfg {
     static constexpr int STAGES = BN == 256 ? 4 : 6;
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
+    static constexpr int OUT_BYTES = EPI_WARPS * 2 * OUT_BOX_BYTES;   // two output boxes per epilogue warp
+    static constexpr int SMEM = STAGES * STAGE_BYTES + OUT_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -77,6 +80,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled:
 // start address, leading offset 16 B (unused by swizzled layouts), 1024 B between 8-row groups,
@@ -189,6 +197,7 @@ struct ChainLayer {
 };
 struct ChainParams {
     CUtensorMap mapX[CHAIN_MAX], mapW[CHAIN_MAX];
+    CUtensorMap mapY[CHAIN_MAX];     // output of a block as 32 x 32 boxes, 64-byte swizzle (unused for the head's last block)
     ChainLayer layer[CHAIN_MAX];
     int first, end;              // blocks [first, end) are computed by this launch
     int depth;                   // blocks of the head: block depth - 1 multiplies by w_out instead of storing
@@ -201,6 +210,7 @@ struct ChainParams {
     uint32_t* status;
 };
 
+__device__ __forceinline__ uint4 ld_residual(const uint4* p, bool past_l1) { return past_l1 ? __ldcg(p) : *p; }
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -224,7 +234,8 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
     unsigned char* aligned = smem_raw + (base - smem_u32(smem_raw));
-    unsigned long long* bars = reinterpret_cast<unsigned long long*>(aligned + C::STAGES * C::STAGE_BYTES);
+    unsigned char* out_stage = aligned + C::STAGES * C::STAGE_BYTES;      // [epilogue warp][2][32 rows][64 bytes]
+    unsigned long long* bars = reinterpret_cast<unsigned long long*>(out_stage + C::OUT_BYTES);
     const uint32_t full0 = smem_u32(bars), empty0 = full0 + 8 * C::STAGES, tfull0 = empty0 + 8 * C::STAGES,
                    tempty0 = tfull0 + 16;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
@@ -330,14 +341,17 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
             const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
             const int m = m0 + q * 32 + lane;
             const bool row_ok = m < P.M;
-            // the residual may have been written by another SM during this launch: read it past L1
+            // The residual was written by other SMs during this launch if l > first.  This SM's L1 can only hold
+            // an older version of those rows if it read the same buffer before it was rewritten, i.e. from the
+            // fourth block of a launch on (two buffers alternate): those reads go past L1.
+            const bool past_l1 = l >= P.first + 3;
             const uint4* xrow = reinterpret_cast<const uint4*>(P.layer[l].X + (size_t)(row_ok ? m : 0) * P.d + n0);
             uint4 xv[4], xn[4];
             mbar_wait(tfull0 + 8 * buf, use, budget);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (warp == 2 && lane == 0) TILE_STAMP(it, 4);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) xn[j] = row_ok ? __ldcg(xrow + (half * CH) * 4 + j) : make_uint4(0, 0, 0, 0);
+            for (int j = 0; j < 4; ++j) xn[j] = row_ok ? ld_residual(xrow + (half * CH) * 4 + j, past_l1) : make_uint4(0, 0, 0, 0);
             float dot = 0.f;
 #pragma unroll 1
             for (int cc = 0; cc < CH; ++cc) {
@@ -348,7 +362,7 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     xv[j] = xn[j];
-                    if (cc + 1 < CH) xn[j] = row_ok ? __ldcg(xrow + (c + 1) * 4 + j) : make_uint4(0, 0, 0, 0);
+                    if (cc + 1 < CH) xn[j] = row_ok ? ld_residual(xrow + (c + 1) * 4 + j, past_l1) : make_uint4(0, 0, 0, 0);
                     bv[j] = bias ? __ldg(reinterpret_cast<const uint4*>(bias + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
                     wv[j] = w_out ? __ldg(reinterpret_cast<const uint4*>(w_out + n0 + c * 32) + j) : make_uint4(0, 0, 0, 0);
                 }
@@ -365,10 +379,20 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
                     const __nv_bfloat162 pk = __floats2bfloat162_rn(y0, y1);
                     out[j] = *reinterpret_cast<const uint32_t*>(&pk);
                 }
-                if (Y && row_ok) {
-                    uint4* yrow = reinterpret_cast<uint4*>(Y + (size_t)m * P.d + n0 + c * 32);
+                if (Y && m0 + q * 32 < P.M) {                  // warp-uniform; rows past M are clipped by the store
+                    // The warp's 32 rows x 64 bytes go to shared memory (64-byte swizzle: 16-byte chunk j of row r
+                    // at chunk j ^ ((r >> 1) & 3), conflict-free) and from there to Y as one TMA store; two boxes
+                    // alternate, a box being rewritten once the store before last has read it.
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+                    unsigned char* box = out_stage + ((warp - 2) * 2 + (cc & 1)) * OUT_BOX_BYTES;
+                    uint4* brow = reinterpret_cast<uint4*>(box + lane * (OUT_COLS * 2));
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) yrow[j] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+                    for (int j = 0; j < 4; ++j)
+                        brow[j ^ ((lane >> 1) & 3)] = make_uint4(out[4 * j], out[4 * j + 1], out[4 * j + 2], out[4 * j + 3]);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) tma_store_2d(&P.mapY[l], smem_u32(box), n0 + c * 32, m0 + q * 32);
                 }
             }
             // this warp has read its part of the accumulator: hand the buffer back to the MMA issuer
@@ -383,6 +407,8 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
             uint32_t* ctr = P.ready + (size_t)l * ntm + t / ntn;
             uint32_t before = 0;
             if (lane == 0) {
+                asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this warp's boxes are written
+                asm volatile("fence.proxy.async;" ::: "memory");            // ... through the async proxy
                 __threadfence();                               // the warp's stores (ordered before by the barrier), then the count
                 before = atomicAdd(ctr, 1u);
             }
@@ -698,29 +724,30 @@ EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// 2-D bf16 row-major [rows, cols] tensor, box {BK, box_rows}, 128-byte swizzle, zero fill outside.
-bool make_map(CUtensorMap* map, const void* ptr, int rows, int cols, int box_rows) {
+// 2-D bf16 row-major [rows, cols] tensor, box {box_cols, box_rows} with rows of 128 bytes (128-byte swizzle) or
+// 64 bytes (64-byte swizzle), zero fill outside.
+bool make_map(CUtensorMap* map, const void* ptr, int rows, int cols, int box_rows, int box_cols) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              CU_TENSOR_MAP_INTERLEAVE_NONE, box_cols * 2 == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // The map of an operand, from the context's cache when this operand has been seen before.  The map is
 // copied out: the next look-up may recycle the slot it came from.
-bool cached_map(specdec_ctx* ctx, CUtensorMap* out, const void* ptr, int rows, int cols, int box_rows) {
+bool cached_map(specdec_ctx* ctx, CUtensorMap* out, const void* ptr, int rows, int cols, int box_rows, int box_cols = BK) {
     static_assert(sizeof(CUtensorMap) <= sizeof(HeadMapEntry::map), "tensor map larger than its cache slot");
     for (HeadMapEntry& e : ctx->head_maps)
-        if (e.ptr == ptr && e.rows == rows && e.cols == cols && e.box_rows == box_rows) {
+        if (e.ptr == ptr && e.rows == rows && e.cols == cols && e.box_rows == box_rows && e.box_cols == box_cols) {
             memcpy(out, e.map, sizeof(CUtensorMap));
             return true;
         }
-    if (!make_map(out, ptr, rows, cols, box_rows)) return false;
+    if (!make_map(out, ptr, rows, cols, box_rows, box_cols)) return false;
     HeadMapEntry& e = ctx->head_maps[ctx->head_map_next];
     ctx->head_map_next = (ctx->head_map_next + 1) % 32;
     memcpy(e.map, out, sizeof(CUtensorMap));
@@ -728,6 +755,7 @@ bool cached_map(specdec_ctx* ctx, CUtensorMap* out, const void* ptr, int rows, i
     e.rows = rows;
     e.cols = cols;
     e.box_rows = box_rows;
+    e.box_cols = box_cols;
     return true;
 }
 
@@ -887,11 +915,18 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
             p.layer[k].X = x;
             p.layer[k].bias = static_cast<const __nv_bfloat16*>(head->b ? head->b[k] : nullptr);
             p.layer[k].Y = k == D - 1 ? nullptr : static_cast<__nv_bfloat16*>(ctx->act[k & 1]);
+            if (p.layer[k].Y) {
+                if (!cached_map(ctx, &p.mapY[k], p.layer[k].Y, (int)M, d, OUT_ROWS, OUT_COLS))
+                    return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
+            } else {
+                p.mapY[k] = p.mapX[0];
+            }
             x = p.layer[k].Y;
         }
         for (int k = D; k < CHAIN_MAX; ++k) {                  // unused slots: defined bytes for the parameter copy
             p.mapX[k] = p.mapX[0];
             p.mapW[k] = p.mapW[0];
+            p.mapY[k] = p.mapX[0];
             p.layer[k] = ChainLayer{nullptr, nullptr, nullptr};
         }
         p.depth = D;

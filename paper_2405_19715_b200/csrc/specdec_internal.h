@@ -10,7 +10,7 @@
 // operand does not pay the driver's encoding again.
 struct HeadMapEntry {
     const void* ptr = nullptr;
-    int rows = 0, cols = 0, box_rows = 0;
+    int rows = 0, cols = 0, box_rows = 0, box_cols = 0;
     alignas(64) unsigned char map[128];
 };
 
@@ -42,7 +42,7 @@ struct specdec_ctx {
     float* head_partial = nullptr;       // [max_B*max_K, max_d/32]
     uint32_t* head_ready = nullptr;      // [8][ceil(max_B*max_K / 128)] finished epilogue warps per (block, 128-row block)
     int head_coop = -1;                  // one cooperative launch for all blocks: -1 not tried, 0 refused (one launch per block), 1 in use
-    HeadMapEntry head_maps[32];          // round-robin cache, keyed by (pointer, rows, cols, box rows)
+    HeadMapEntry head_maps[32];          // round-robin cache, keyed by (pointer, rows, cols, box rows, box cols)
     int head_map_next = 0;
     char err[256] = "no error";
 };
