@@ -204,7 +204,9 @@ struct ChainParams {
     int M, d;
     const __nv_bfloat16* w_out;  // [d]
     float* partial;              // [M, 2 * d / BN] partial dots of the last block
-    uint32_t* ready;             // [depth][row blocks] epilogue warps that have finished a tile of (block, row block)
+    uint32_t* ready;             // [depth][row blocks] epilogue warps that have finished a tile of (block, row block); zero at launch
+    uint32_t* ready_next;        // the next call's counters, cleared by this launch (a call that gave up leaves no trace either)
+    int ready_words;
     float* accept_prob;
     float b_out;
     uint32_t* status;
@@ -241,6 +243,8 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (blockIdx.x == gridDim.x - 1)
+        for (int i = tid; i < P.ready_words; i += HEAD_THREADS) P.ready_next[i] = 0;
     const int nkb = P.d / BK;
     const int ntn = P.d / BN, ntm = (P.M + BM - 1) / BM, per_block = ntn * ntm;
     const int ntiles = (P.end - P.first) * per_block;
@@ -934,13 +938,15 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
         p.d = d;
         p.w_out = static_cast<const __nv_bfloat16*>(head->w_out);
         p.partial = ctx->head_partial;
-        p.ready = ctx->head_ready;
+        const size_t set_words = (size_t)CHAIN_MAX * (((size_t)ctx->max_B * ctx->max_K + BM - 1) / BM);
+        p.ready = ctx->head_ready + (size_t)ctx->head_ready_set * set_words;
+        ctx->head_ready_set ^= 1;
+        p.ready_next = ctx->head_ready + (size_t)ctx->head_ready_set * set_words;
+        p.ready_words = (int)set_words;
         p.accept_prob = accept_prob;
         p.b_out = head->b_out;
         p.status = ctx->status;
-        const size_t ntm = (size_t)((M + BM - 1) / BM);
-        cudaError_t e = cudaMemsetAsync(ctx->head_ready, 0, (size_t)D * ntm * sizeof(uint32_t), s);
-        if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
+        cudaError_t e = cudaSuccess;
         auto launch = [&](int first, int end, bool coop) {
             return BN == 256 ? launch_chain<256>(p, first, end, ctx->sm_count, coop, s)
                              : launch_chain<128>(p, first, end, ctx->sm_count, coop, s);
