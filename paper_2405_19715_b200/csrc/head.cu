@@ -30,11 +30,13 @@ constexpr uint32_t WAIT_POLLS = 1u << 24;
 constexpr int OUT_COLS = 32, OUT_ROWS = 32;                       // box of one TMA store of the output: 32 rows x 64 bytes
 constexpr int OUT_BOX_BYTES = OUT_ROWS * OUT_COLS * 2;
 
-template <int BN> struct Cfg {
-    static constexpr int STAGES = BN == 256 ? 4 : 6;
+// PAIR: two CTAs (a cluster) share a 256 x BN tile; each loads its 128 rows of X and its half of the tile's
+// weight rows, and one thread of the even CTA issues M = 256 MMAs over both CTAs' shared and tensor memory.
+template <int BN, bool PAIR> struct Cfg {
     static constexpr int A_BYTES = BM * BK * 2;
-    static constexpr int B_BYTES = BN * BK * 2;
+    static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = 192 * 1024 / STAGE_BYTES;           // 4 stages of 48 KB, 6 of 32 KB, 8 of 24 KB
     static constexpr int OUT_BYTES = EPI_WARPS * 2 * OUT_BOX_BYTES;   // two output boxes per epilogue warp
     static constexpr int SMEM = STAGES * STAGE_BYTES + OUT_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 };
@@ -130,6 +132,58 @@ __device__ __forceinline__ void umma_kblock(uint32_t tmem_d, uint32_t a_lo, uint
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// ---- the same for a pair of CTAs (cta_group::2) ----
+__device__ __forceinline__ uint32_t pair_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void pair_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The address of this CTA's shared-memory location `a` in CTA `rank` of the pair.
+__device__ __forceinline__ uint32_t pair_map(uint32_t a, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(rank));
+    return r;
+}
+// TMA load by one CTA of a pair whose bytes are counted on the EVEN CTA's barrier (peer bit of the barrier's
+// cluster address cleared).  No multicast: each CTA fetches its own operands.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar & 0xFEFFFFFFu) : "memory");
+}
+__device__ __forceinline__ void umma_kblock_pair(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc_first) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t.reg .b32 ta, tb;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "setp.eq.b32 q, 0, 0;\n\t"
+        "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t"
+        "add.u32 ta, %1, 2;\n\tadd.u32 tb, %2, 2;\n\t"
+        "mov.b64 da, {ta, %5};\n\tmov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, q;\n\t"
+        "add.u32 ta, %1, 4;\n\tadd.u32 tb, %2, 4;\n\t"
+        "mov.b64 da, {ta, %5};\n\tmov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, q;\n\t"
+        "add.u32 ta, %1, 6;\n\tadd.u32 tb, %2, 6;\n\t"
+        "mov.b64 da, {ta, %5};\n\tmov.b64 db, {tb, %5};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, q;\n\t}"
+        ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(acc_first), "r"(UMMA_DESC_HI) : "memory");
+}
+// Arrive on the barrier at this offset in both CTAs of the pair once the pair's MMAs issued so far have completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+__host__ __device__ constexpr uint32_t umma_idesc_pair(int n) {           // M = 256 across the pair
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     uint32_t r[32];
@@ -229,10 +283,10 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
 // operands with nothing to overlap.  The accumulator is double-buffered in tensor memory (2 x BN columns), so
 // the epilogue of one tile runs while the MMAs of the next are issued.  In the head's last block the warp that
 // completes a row block's count adds the block's partial dots in column order and applies the sigmoid.
-template <int BN>
+template <int BN, bool PAIR>
 __global__ void __launch_bounds__(HEAD_THREADS, 1)
 head_chain_kernel(const __grid_constant__ ChainParams P) {
-    using C = Cfg<BN>;
+    using C = Cfg<BN, PAIR>;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
     unsigned char* aligned = smem_raw + (base - smem_u32(smem_raw));
@@ -245,8 +299,13 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (blockIdx.x == gridDim.x - 1)
         for (int i = tid; i < P.ready_words; i += HEAD_THREADS) P.ready_next[i] = 0;
+    constexpr int TM = PAIR ? 2 * BM : BM;                                // rows of a tile
+    const uint32_t rank = PAIR ? pair_rank() : 0u;                        // 0: issues the pair's MMAs, owns its barriers
+    const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;   // a CTA or a pair of CTAs
+    const int nworkers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     const int nkb = P.d / BK;
-    const int ntn = P.d / BN, ntm = (P.M + BM - 1) / BM, per_block = ntn * ntm;
+    const int ntn = P.d / BN, ntm = (P.M + TM - 1) / TM, per_block = ntn * ntm;
+    const int nrb = ntm * (TM / BM);                                      // 128-row blocks with a counter (the last may be empty)
     const int ntiles = (P.end - P.first) * per_block;
     const uint32_t tile_warps = (uint32_t)(ntn * EPI_WARPS);              // counts that complete a row block
     uint32_t budget = WAIT_POLLS;
@@ -258,18 +317,25 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(tfull0 + 8 * b, 1);
-            mbar_init(tempty0 + 8 * b, EPI_WARPS);
+            mbar_init(tempty0 + 8 * b, PAIR ? 2 * EPI_WARPS : EPI_WARPS);   // a pair: the even CTA's, for both epilogues
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {                      // this warp owns the tensor-memory allocation
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)(2 * BN)) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (warp == 1) {                      // this warp owns the tensor-memory allocation (of a pair: the same warp of both CTAs)
+        if constexpr (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)(2 * BN)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)(2 * BN)) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if constexpr (PAIR) pair_sync();      // both CTAs' barriers exist before anything is sent to them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(tmem_slot);
 
@@ -277,11 +343,12 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, it = 0;
-            for (int g = blockIdx.x; g < ntiles; g += gridDim.x, ++it) {
+            for (int g = worker; g < ntiles; g += nworkers, ++it) {
                 const int l = P.first + g / per_block, t = g % per_block;
-                const int m0 = (t / ntn) * BM, n0 = (t % ntn) * BN;
+                const int m0 = (t / ntn) * TM + (int)rank * BM;                         // this CTA's rows of X
+                const int n0 = (t % ntn) * BN + (PAIR ? (int)rank * (BN / 2) : 0);      // ... and rows of W
                 if (l > P.first) {                             // the rows of X come from this launch's previous block
-                    const uint32_t* ctr = P.ready + (size_t)(l - 1) * ntm + t / ntn;
+                    const uint32_t* ctr = P.ready + (size_t)(l - 1) * nrb + m0 / BM;
                     uint32_t polls = 0;
                     while (ld_acquire_u32(ctr) < tile_warps)
                         if (++polls >= (budget == WAIT_POLLS ? FLAG_POLLS : WAIT_POLLS_LEFT)) {
@@ -296,21 +363,27 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
                     mbar_wait(empty0 + 8 * stage, phase ^ 1u, budget);
                     if (kb == 0) TILE_STAMP(it, 0);
                     const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
-                    mbar_expect_tx(full0 + 8 * stage, C::STAGE_BYTES);
-                    tma_load_2d(a, mx, kb * BK, m0, full0 + 8 * stage);
-                    tma_load_2d(b, mw, kb * BK, n0, full0 + 8 * stage);
+                    if constexpr (PAIR) {                      // both CTAs' bytes complete the even CTA's barrier
+                        if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * C::STAGE_BYTES);
+                        tma_load_2d_pair(a, mx, kb * BK, m0, full0 + 8 * stage);
+                        tma_load_2d_pair(b, mw, kb * BK, n0, full0 + 8 * stage);
+                    } else {
+                        mbar_expect_tx(full0 + 8 * stage, C::STAGE_BYTES);
+                        tma_load_2d(a, mx, kb * BK, m0, full0 + 8 * stage);
+                        tma_load_2d(b, mw, kb * BK, n0, full0 + 8 * stage);
+                    }
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc(BN);
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = PAIR ? umma_idesc_pair(BN) : umma_idesc(BN);
             static_assert(BK / UMMA_K == 4, "umma_kblock issues four MMAs");
             const uint32_t desc_lo0 = umma_desc_lo(base);      // stage 0 of the ring, operand A, k = 0
             uint32_t stage = 0, phase = 0, it = 0;
-            for (int g = blockIdx.x; g < ntiles; g += gridDim.x, ++it) {
+            for (int g = worker; g < ntiles; g += nworkers, ++it) {
                 const uint32_t buf = it & 1u, use = (it >> 1) & 1u;
                 mbar_wait(tempty0 + 8 * buf, use ^ 1u, budget);      // epilogue has drained this accumulator
                 TILE_STAMP(it, 1);
@@ -321,11 +394,17 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
                     if (kb == 0) TILE_STAMP(it, 2);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_lo = desc_lo0 + stage * (C::STAGE_BYTES >> 4);
-                    umma_kblock(acc, a_lo, a_lo + (C::A_BYTES >> 4), idesc, kb != 0 ? 1u : 0u);
-                    umma_commit(empty0 + 8 * stage);          // stage reusable once these MMAs have read it
+                    if constexpr (PAIR) {
+                        umma_kblock_pair(acc, a_lo, a_lo + (C::A_BYTES >> 4), idesc, kb != 0 ? 1u : 0u);
+                        umma_commit_pair(empty0 + 8 * stage);  // stage reusable, in both CTAs, once these MMAs have read it
+                    } else {
+                        umma_kblock(acc, a_lo, a_lo + (C::A_BYTES >> 4), idesc, kb != 0 ? 1u : 0u);
+                        umma_commit(empty0 + 8 * stage);
+                    }
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                 }
-                umma_commit(tfull0 + 8 * buf);                // accumulator complete
+                if constexpr (PAIR) umma_commit_pair(tfull0 + 8 * buf);   // accumulator complete (in both CTAs)
+                else umma_commit(tfull0 + 8 * buf);
                 TILE_STAMP(it, 3);
             }
         }
@@ -335,9 +414,9 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
         const int half = (warp - 2) >> 2;                  // which half of the tile's columns
         constexpr int CH = BN / 32 / 2;                    // 32-column chunks per warp
         uint32_t it = 0;
-        for (int g = blockIdx.x; g < ntiles; g += gridDim.x, ++it) {
+        for (int g = worker; g < ntiles; g += nworkers, ++it) {
             const int l = P.first + g / per_block, t = g % per_block;
-            const int m0 = (t / ntn) * BM, n0 = (t % ntn) * BN;
+            const int m0 = (t / ntn) * TM + (int)rank * BM, n0 = (t % ntn) * BN;
             const bool last = l == P.depth - 1;
             const __nv_bfloat16* bias = P.layer[l].bias;
             const __nv_bfloat16* w_out = last ? P.w_out : nullptr;
@@ -402,13 +481,16 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
             // this warp has read its part of the accumulator: hand the buffer back to the MMA issuer
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty0 + 8 * buf);
+            if (lane == 0) {
+                if (PAIR && rank != 0) mbar_arrive_cluster(pair_map(tempty0 + 8 * buf, 0));
+                else mbar_arrive(tempty0 + 8 * buf);
+            }
             if (warp == 2 && lane == 0) TILE_STAMP(it, 5);
             if (last && row_ok) P.partial[(size_t)m * (2 * ntn) + 2 * (t % ntn) + half] = dot;
             // count this warp's part of the tile as written; the count of a row block is what the next block's
             // tiles (their TMA loads: the async proxy) and, in the last block, the row block's finisher wait for
             __syncwarp();
-            uint32_t* ctr = P.ready + (size_t)l * ntm + t / ntn;
+            uint32_t* ctr = P.ready + (size_t)l * nrb + m0 / BM;
             uint32_t before = 0;
             if (lane == 0) {
                 asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // this warp's boxes are written
@@ -433,9 +515,13 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
     report_wait_limit(P.status, budget);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if constexpr (PAIR) pair_sync();      // nothing is in flight towards the other CTA's barriers or tensor memory any more
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)(2 * BN)) : "memory");
+        if constexpr (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)(2 * BN)) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)(2 * BN)) : "memory");
     }
 }
 
@@ -803,37 +889,102 @@ cudaError_t launch_swap(const CUtensorMap& mx, const CUtensorMap& mw, const Bloc
 }
 
 // Blocks [first, end) of the chain in one launch; cooperative when it spans more than one block (its CTAs
-// then wait for one another's tiles and must all be resident).
-template <int BN>
+// then wait for one another's tiles and must all be resident).  PAIR: clusters of two CTAs, one 256-row tile each.
+template <int BN, bool PAIR>
 cudaError_t launch_chain(ChainParams& p, int first, int end, int sm_count, bool cooperative, cudaStream_t s) {
+    using C = Cfg<BN, PAIR>;
     static unsigned long long allowed = 0;                                // per device: large dynamic shared memory granted
     int dev = 0;
     cudaGetDevice(&dev);
     if (!((allowed >> (dev & 63)) & 1ull)) {
-        cudaError_t e = cudaFuncSetAttribute(head_chain_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::SMEM);
+        cudaError_t e = cudaFuncSetAttribute(head_chain_kernel<BN, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
         if (e != cudaSuccess) return e;
         allowed |= 1ull << (dev & 63);
     }
     p.first = first;
     p.end = end;
-    const int ntiles = (end - first) * (p.d / BN) * ((p.M + BM - 1) / BM);
+    constexpr int TM = PAIR ? 2 * BM : BM;
+    const int ntiles = (end - first) * (p.d / BN) * ((p.M + TM - 1) / TM);
+    const int workers = std::min(ntiles, PAIR ? sm_count / 2 : sm_count);  // one CTA per SM (its ring fills the shared memory)
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)std::min(ntiles, sm_count));             // one CTA per SM (its ring fills the shared memory)
+    cfg.gridDim = dim3((unsigned)(PAIR ? 2 * workers : workers));
     cfg.blockDim = dim3(HEAD_THREADS);
-    cfg.dynamicSmemBytes = (size_t)Cfg<BN>::SMEM;
+    cfg.dynamicSmemBytes = (size_t)C::SMEM;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = cooperative ? 1 : 0;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, head_chain_kernel<BN>, p);
+    cfg.numAttrs = PAIR ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, head_chain_kernel<BN, PAIR>, p);
 }
 
 int fail(specdec_ctx* ctx, int code, const char* msg) {
     snprintf(ctx->err, sizeof(ctx->err), "%s", msg);
     return code;
 }
+
+// One call of the head for more than 256 rows: all D blocks as tiles of one launch (`coop`) or one launch per block.
+cudaError_t launch_chain_call(specdec_ctx* ctx, const __nv_bfloat16* x, const specdec_head* head, int M, int d, int D, int BN,
+                              float* accept_prob, bool pair, bool coop, cudaStream_t s) {
+    ChainParams p = {};
+    for (int k = 0; k < D; ++k) {
+        if (!cached_map(ctx, &p.mapX[k], x, M, d, BM) || !cached_map(ctx, &p.mapW[k], head->W[k], d, d, pair ? BN / 2 : BN))
+            return cudaErrorUnknown;
+        p.layer[k].X = x;
+        p.layer[k].bias = static_cast<const __nv_bfloat16*>(head->b ? head->b[k] : nullptr);
+        p.layer[k].Y = k == D - 1 ? nullptr : static_cast<__nv_bfloat16*>(ctx->act[k & 1]);
+        if (p.layer[k].Y) {
+            if (!cached_map(ctx, &p.mapY[k], p.layer[k].Y, M, d, OUT_ROWS, OUT_COLS)) return cudaErrorUnknown;
+        } else {
+            p.mapY[k] = p.mapX[0];
+        }
+        x = p.layer[k].Y;
+    }
+    for (int k = D; k < CHAIN_MAX; ++k) {                      // unused slots: defined bytes for the parameter copy
+        p.mapX[k] = p.mapX[0];
+        p.mapW[k] = p.mapW[0];
+        p.mapY[k] = p.mapX[0];
+        p.layer[k] = ChainLayer{nullptr, nullptr, nullptr};
+    }
+    p.depth = D;
+    p.M = M;
+    p.d = d;
+    p.w_out = static_cast<const __nv_bfloat16*>(head->w_out);
+    p.partial = ctx->head_partial;
+    const size_t set_words = (size_t)CHAIN_MAX * (((size_t)ctx->max_B * ctx->max_K + BM - 1) / BM + 1);
+    p.ready = ctx->head_ready + (size_t)ctx->head_ready_set * set_words;
+    p.ready_next = ctx->head_ready + (size_t)(ctx->head_ready_set ^ 1) * set_words;
+    p.ready_words = (int)set_words;
+    p.accept_prob = accept_prob;
+    p.b_out = head->b_out;
+    p.status = ctx->status;
+    auto launch = [&](int first, int end) {
+        if (pair)
+            return BN == 256 ? launch_chain<256, true>(p, first, end, ctx->sm_count, coop, s)
+                             : launch_chain<128, true>(p, first, end, ctx->sm_count, coop, s);
+        return BN == 256 ? launch_chain<256, false>(p, first, end, ctx->sm_count, coop, s)
+                         : launch_chain<128, false>(p, first, end, ctx->sm_count, coop, s);
+    };
+    if (coop) {
+        const cudaError_t e = launch(0, D);
+        if (e != cudaSuccess) return e;
+        ctx->launches += 1;
+    } else {
+        for (int k = 0; k < D; ++k) {
+            const cudaError_t e = launch(k, k + 1);
+            if (e != cudaSuccess) return e;             // after a first block was enqueued: a real error, not a refused configuration
+            ctx->launches += 1;
+        }
+    }
+    ctx->head_ready_set ^= 1;                                  // the sets change roles only when something was launched
+    return cudaSuccess;
+}
+
 
 }  // namespace
 
@@ -912,63 +1063,21 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
             x = p.Y;
         }
     } else {
-        ChainParams p;
-        for (int k = 0; k < D; ++k) {
-            if (!cached_map(ctx, &p.mapX[k], x, (int)M, d, BM) || !cached_map(ctx, &p.mapW[k], head->W[k], d, d, BN))
-                return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
-            p.layer[k].X = x;
-            p.layer[k].bias = static_cast<const __nv_bfloat16*>(head->b ? head->b[k] : nullptr);
-            p.layer[k].Y = k == D - 1 ? nullptr : static_cast<__nv_bfloat16*>(ctx->act[k & 1]);
-            if (p.layer[k].Y) {
-                if (!cached_map(ctx, &p.mapY[k], p.layer[k].Y, (int)M, d, OUT_ROWS, OUT_COLS))
-                    return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
-            } else {
-                p.mapY[k] = p.mapX[0];
-            }
-            x = p.layer[k].Y;
-        }
-        for (int k = D; k < CHAIN_MAX; ++k) {                  // unused slots: defined bytes for the parameter copy
-            p.mapX[k] = p.mapX[0];
-            p.mapW[k] = p.mapW[0];
-            p.mapY[k] = p.mapX[0];
-            p.layer[k] = ChainLayer{nullptr, nullptr, nullptr};
-        }
-        p.depth = D;
-        p.M = (int)M;
-        p.d = d;
-        p.w_out = static_cast<const __nv_bfloat16*>(head->w_out);
-        p.partial = ctx->head_partial;
-        const size_t set_words = (size_t)CHAIN_MAX * (((size_t)ctx->max_B * ctx->max_K + BM - 1) / BM);
-        p.ready = ctx->head_ready + (size_t)ctx->head_ready_set * set_words;
-        ctx->head_ready_set ^= 1;
-        p.ready_next = ctx->head_ready + (size_t)ctx->head_ready_set * set_words;
-        p.ready_words = (int)set_words;
-        p.accept_prob = accept_prob;
-        p.b_out = head->b_out;
-        p.status = ctx->status;
-        cudaError_t e = cudaSuccess;
-        auto launch = [&](int first, int end, bool coop) {
-            return BN == 256 ? launch_chain<256>(p, first, end, ctx->sm_count, coop, s)
-                             : launch_chain<128>(p, first, end, ctx->sm_count, coop, s);
-        };
-        if (ctx->head_coop != 0 && D > 1) {
-            e = launch(0, D, true);
-            if (e == cudaSuccess) {
-                ctx->head_coop = 1;
-                ctx->launches += 1;
-            } else if (ctx->head_coop < 0 && (e == cudaErrorCooperativeLaunchTooLarge || e == cudaErrorNotSupported)) {
-                (void)cudaGetLastError();                          // this device or partition cannot hold the grid: one launch per block
-                ctx->head_coop = 0;
-            } else {
-                return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
-            }
-        }
-        if (ctx->head_coop == 0 || D == 1) {
-            for (int k = 0; k < D; ++k) {
-                e = launch(k, k + 1, false);
-                if (e != cudaSuccess) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
-                ctx->launches += 1;
-            }
+        // Preferred: a pair of CTAs per 256-row tile (a third less operand traffic per SM) and all blocks in one
+        // cooperative launch.  A device or partition that refuses clusters or the cooperative grid gets one CTA
+        // per tile, then one launch per block; what was refused is remembered in the context.
+        for (;;) {
+            const bool pair = ctx->head_pair != 0 && ctx->sm_count >= 2;
+            const bool coop = ctx->head_coop != 0 && D > 1;
+            cudaError_t e = launch_chain_call(ctx, x, head, (int)M, d, D, BN, accept_prob, pair, coop, s);
+            if (e == cudaSuccess) break;
+            const bool config_error = e == cudaErrorCooperativeLaunchTooLarge || e == cudaErrorNotSupported ||
+                                      e == cudaErrorInvalidValue || e == cudaErrorInvalidConfiguration ||
+                                      e == cudaErrorLaunchOutOfResources;
+            if (!config_error || (!pair && !coop)) return fail(ctx, SPECDEC_ECUDA, cudaGetErrorString(e));
+            (void)cudaGetLastError();
+            if (pair) ctx->head_pair = 0;
+            else ctx->head_coop = 0;
         }
     }
     cudaError_t e = cudaGetLastError();
