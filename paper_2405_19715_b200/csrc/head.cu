@@ -35,8 +35,12 @@ constexpr int OUT_BOX_BYTES = OUT_ROWS * OUT_COLS * 2;
 template <int BN, bool PAIR> struct Cfg {
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;
-    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = 192 * 1024 / STAGE_BYTES;           // 4 stages of 48 KB, 6 of 32 KB, 8 of 24 KB
+    static constexpr int KB_BYTES = A_BYTES + B_BYTES;                // operands of one k-block
+    // k-blocks per ring stage, i.e. per barrier round trip of the issuing thread: with the pair's smaller operands
+    // two k-blocks (eight MMAs) share one wait and one commit and the ring still holds three stages
+    static constexpr int KSUB = PAIR ? 2 : 1;
+    static constexpr int STAGE_BYTES = KSUB * KB_BYTES;
+    static constexpr int STAGES = 192 * 1024 / STAGE_BYTES;           // 4 x 48 KB or 6 x 32 KB; pairs: 3 x 64 KB or 4 x 48 KB
     static constexpr int OUT_BYTES = EPI_WARPS * 2 * OUT_BOX_BYTES;   // two output boxes per epilogue warp
     static constexpr int SMEM = STAGES * STAGE_BYTES + OUT_BYTES + 1024 /* alignment slack */ + 256 /* barriers */;
 };
@@ -359,18 +363,25 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
                 }
                 const CUtensorMap* mx = &P.mapX[l];
                 const CUtensorMap* mw = &P.mapW[l];
-                for (int kb = 0; kb < nkb; ++kb) {
+                for (int ks = 0; ks < nkb / C::KSUB; ++ks) {
                     mbar_wait(empty0 + 8 * stage, phase ^ 1u, budget);
-                    if (kb == 0) TILE_STAMP(it, 0);
-                    const uint32_t a = base + stage * C::STAGE_BYTES, b = a + C::A_BYTES;
+                    if (ks == 0) TILE_STAMP(it, 0);
                     if constexpr (PAIR) {                      // both CTAs' bytes complete the even CTA's barrier
                         if (rank == 0) mbar_expect_tx(full0 + 8 * stage, 2 * C::STAGE_BYTES);
-                        tma_load_2d_pair(a, mx, kb * BK, m0, full0 + 8 * stage);
-                        tma_load_2d_pair(b, mw, kb * BK, n0, full0 + 8 * stage);
                     } else {
                         mbar_expect_tx(full0 + 8 * stage, C::STAGE_BYTES);
-                        tma_load_2d(a, mx, kb * BK, m0, full0 + 8 * stage);
-                        tma_load_2d(b, mw, kb * BK, n0, full0 + 8 * stage);
+                    }
+#pragma unroll
+                    for (int h = 0; h < C::KSUB; ++h) {
+                        const uint32_t a = base + stage * C::STAGE_BYTES + h * C::KB_BYTES, b = a + C::A_BYTES;
+                        const int k0 = (ks * C::KSUB + h) * BK;
+                        if constexpr (PAIR) {
+                            tma_load_2d_pair(a, mx, k0, m0, full0 + 8 * stage);
+                            tma_load_2d_pair(b, mw, k0, n0, full0 + 8 * stage);
+                        } else {
+                            tma_load_2d(a, mx, k0, m0, full0 + 8 * stage);
+                            tma_load_2d(b, mw, k0, n0, full0 + 8 * stage);
+                        }
                     }
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -389,18 +400,18 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
                 TILE_STAMP(it, 1);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t acc = tmem + buf * BN;
-                for (int kb = 0; kb < nkb; ++kb) {
+                for (int ks = 0; ks < nkb / C::KSUB; ++ks) {
                     mbar_wait(full0 + 8 * stage, phase, budget);
-                    if (kb == 0) TILE_STAMP(it, 2);
+                    if (ks == 0) TILE_STAMP(it, 2);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a_lo = desc_lo0 + stage * (C::STAGE_BYTES >> 4);
-                    if constexpr (PAIR) {
-                        umma_kblock_pair(acc, a_lo, a_lo + (C::A_BYTES >> 4), idesc, kb != 0 ? 1u : 0u);
-                        umma_commit_pair(empty0 + 8 * stage);  // stage reusable, in both CTAs, once these MMAs have read it
-                    } else {
-                        umma_kblock(acc, a_lo, a_lo + (C::A_BYTES >> 4), idesc, kb != 0 ? 1u : 0u);
-                        umma_commit(empty0 + 8 * stage);
+#pragma unroll
+                    for (int h = 0; h < C::KSUB; ++h) {
+                        const uint32_t a_lo = desc_lo0 + stage * (C::STAGE_BYTES >> 4) + h * (C::KB_BYTES >> 4);
+                        if constexpr (PAIR) umma_kblock_pair(acc, a_lo, a_lo + (C::A_BYTES >> 4), idesc, (ks | h) != 0 ? 1u : 0u);
+                        else umma_kblock(acc, a_lo, a_lo + (C::A_BYTES >> 4), idesc, (ks | h) != 0 ? 1u : 0u);
                     }
+                    if constexpr (PAIR) umma_commit_pair(empty0 + 8 * stage);   // stage reusable, in both CTAs, once these MMAs have read it
+                    else umma_commit(empty0 + 8 * stage);
                     if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if constexpr (PAIR) umma_commit_pair(tfull0 + 8 * buf);   // accumulator complete (in both CTAs)
