@@ -103,6 +103,14 @@ int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits);
 /* Number of kernels this context has launched so far (for launch accounting). */
 uint64_t specdec_launch_count(const specdec_ctx* ctx);
 
+/* How specdec_accept_head launches the residual blocks (Eq. 3) when B*K > 256.  By default the call tries, and
+ * remembers per context what the device accepted: a pair of CTAs (thread-block cluster of two) per 256-row tile
+ * and all blocks in one cooperative launch; without clusters one CTA per 128-row tile; without a cooperative
+ * grid one launch per block.  pair = 0 / cooperative = 0 rule the respective form out for this context from now
+ * on (a partition on which it should not be tried; tests of the fallbacks); 1 allows it again.  Results are the
+ * same in every form up to the summation order inside a tile, which does not change.  Host only; no GPU work. */
+int specdec_head_launch_mode(specdec_ctx* ctx, int pair, int cooperative);
+
 /* Synchronises `stream`; *logit_rows receives the number of logit rows (V elements each: two per candidate
  * position, one for a bonus position) that units leaving early under SPECDEC_VERIFY_EARLY_EXIT did not read
  * since the last call of this function (the counter is then cleared). */

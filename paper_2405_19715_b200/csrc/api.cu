@@ -165,6 +165,13 @@ int specdec_set_phase_stamps(specdec_ctx* ctx, uint64_t* stamps, size_t units) {
 #endif
 }
 
+int specdec_head_launch_mode(specdec_ctx* ctx, int pair, int cooperative) {
+    if (!ctx) return SPECDEC_EINVAL;
+    ctx->head_pair = pair ? 1 : 0;
+    ctx->head_coop = cooperative ? -1 : 0;                 // -1: allowed, not yet confirmed by a launch
+    return SPECDEC_OK;
+}
+
 int specdec_device_status(specdec_ctx* ctx, void* stream, uint32_t* bits) {
     if (!ctx) return SPECDEC_EINVAL;
     if (int rc = specdec_use_device(ctx)) return rc;

@@ -44,7 +44,7 @@ struct specdec_ctx {
                                          // counts in one of the two sets and clears the other for the next call
     int head_ready_set = 0;
     int head_pair = 1;                   // a pair of CTAs per 256-row tile (0: one CTA per 128-row tile)
-    int head_coop = -1;                  // one cooperative launch for all blocks: -1 not tried, 0 refused (one launch per block), 1 in use
+    int head_coop = -1;                  // one cooperative launch for all blocks: 0 ruled out or refused (one launch per block)
     HeadMapEntry head_maps[32];          // round-robin cache, keyed by (pointer, rows, cols, box rows, box cols)
     int head_map_next = 0;
     char err[256] = "no error";

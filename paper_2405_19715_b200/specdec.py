@@ -19,7 +19,7 @@ DATA_BAD_LENGTH, DATA_BAD_TOKEN, DATA_WAIT_LIMIT, DATA_TOPK_TIES = 1, 2, 4, 8
 VERIFY_EARLY_EXIT = 0x100
 
 EXPORTS = ["specdec_create", "specdec_destroy", "specdec_last_error", "specdec_device_status",
-           "specdec_launch_count", "specdec_last_kernel", "specdec_set_phase_stamps", "specdec_early_exit_count", "specdec_verify_correct", "specdec_verify_correct_host",
+           "specdec_launch_count", "specdec_last_kernel", "specdec_set_phase_stamps", "specdec_early_exit_count", "specdec_head_launch_mode", "specdec_verify_correct", "specdec_verify_correct_host",
            "specdec_accept_head", "specdec_stop", "specdec_verify_correct_static", "specdec_verify_greedy", "specdec_stop_step", "specdec_selftest_wait_limit", "specdec_verify_correct_topk", "specdec_sample",
            "specdec_shard_stats", "specdec_shard_accept", "specdec_shard_draw"]
 SHARD_STATS_WIDTH, SHARD_MAX_RANKS = 8, 64
@@ -65,6 +65,7 @@ def load_library(path: str | Path | None = None) -> C.CDLL:
     lib.specdec_last_kernel.argtypes = [C.c_void_p]
     lib.specdec_last_kernel.restype = C.c_char_p
     lib.specdec_set_phase_stamps.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t]
+    lib.specdec_head_launch_mode.argtypes = [C.c_void_p, C.c_int, C.c_int]
     lib.specdec_early_exit_count.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_uint64)]
     lib.specdec_verify_correct.argtypes = [C.c_void_p, vp, vp, C.c_int, ip, ip, fp, C.c_float, C.c_int, C.c_int,
                                            C.c_int, ip, ip, fp, fp, fp, C.c_uint32, C.c_void_p]
@@ -176,6 +177,11 @@ class Context:
             self._check(self.lib.specdec_set_phase_stamps(self.handle, None, 0))
         else:
             self._check(self.lib.specdec_set_phase_stamps(self.handle, _ptr(stamps, torch.int64), stamps.shape[0]))
+
+    def head_launch_mode(self, pair: bool = True, cooperative: bool = True):
+        """specdec_head_launch_mode of the C ABI: rule out (False) or allow the pair-of-CTAs tiles and the single
+        cooperative launch of the acceptance head for more than 256 rows."""
+        self._check(self.lib.specdec_head_launch_mode(self.handle, int(pair), int(cooperative)))
 
     def early_exit_count(self, stream=None) -> int:
         """specdec_early_exit_count of the C ABI: logit rows left unread by early exits since the last call (synchronises)."""

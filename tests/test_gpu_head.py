@@ -73,6 +73,32 @@ def test_head_many_row_tiles(rows, d, depth):
     ctx.close()
 
 
+
+@pytest.mark.parametrize("rows,d,depth", [((30, 20), 384, 3), ((75, 40), 768, 4), ((9, 33), 512, 2)],
+                         ids=["600x384x3", "3000x768x4", "297x512x2"])
+def test_head_launch_forms_agree(rows, d, depth):
+    """The three forms specdec_accept_head falls back through for more than 256 rows -- pairs of CTAs in one
+    cooperative launch, one CTA per tile in one cooperative launch, one launch per block (with and without
+    pairs) -- each against the oracle and against one another (the arithmetic per output is the same)."""
+    B, K = rows
+    ctx = specdec.Context(B, K, max_d=d)
+    hidden, Ws, bs, w_out, b_out = _head_problem(900 + d + depth, B, K, d, depth, True, std=0.02)
+    want = orc.accept_head(hidden, list(zip(Ws, bs)), w_out, b_out)
+    outs = {}
+    for pair in (True, False):
+        for coop in (True, False):
+            ctx.head_launch_mode(pair=pair, cooperative=coop)
+            n0 = ctx.launch_count()
+            got = _run_head(ctx, hidden, Ws, bs, w_out, b_out)
+            assert ctx.launch_count() - n0 == (1 if coop else depth), (pair, coop)
+            err = np.abs(got - want) / want
+            assert err.max() <= HEAD_RTOL, (pair, coop, err.max())
+            outs[(pair, coop)] = got
+    ref = outs[(True, True)]
+    for key, got in outs.items():
+        np.testing.assert_allclose(got, ref, rtol=1e-5, atol=0, err_msg=str(key))
+    ctx.close()
+
 @pytest.mark.parametrize("rows", [1, 2, 3, 4, 5, 8, 9, 13, 16, 17, 32, 33, 64, 65])
 @pytest.mark.parametrize("d,depth,with_bias", [(256, 1, True), (512, 3, False), (4096, 2, True)])
 def test_head_few_rows(rows, d, depth, with_bias):
