@@ -98,7 +98,7 @@ int specdec_create(specdec_ctx** out, int device, int max_B, int max_K, int max_
             e = cudaMalloc(&ctx->head_partial, (size_t)max_B * max_K * ((max_d + 31) / 32) * sizeof(float));
         if (e == cudaSuccess)
         {
-            const size_t n = 2 * 8 * (((size_t)max_B * max_K + 127) / 128 + 1) * sizeof(uint32_t);
+            const size_t n = (1 + 8 * (((size_t)max_B * max_K + 127) / 128 + 1)) * sizeof(uint32_t);
             e = cudaMalloc(&ctx->head_ready, n);
             if (e == cudaSuccess) e = cudaMemset(ctx->head_ready, 0, n);
         }

@@ -262,9 +262,9 @@ struct ChainParams {
     int M, d;
     const __nv_bfloat16* w_out;  // [d]
     float* partial;              // [M, 2 * d / BN] partial dots of the last block
-    uint32_t* ready;             // [depth][row blocks] epilogue warps that have finished a tile of (block, row block); zero at launch
-    uint32_t* ready_next;        // the next call's counters, cleared by this launch (a call that gave up leaves no trace either)
-    int ready_words;
+    uint32_t* ready;             // [depth][row blocks] epilogue warps that have finished a tile of (block, row block); zero at
+                                 // launch, and cleared again by the CTA that leaves last (so a launch may be replayed from a graph)
+    uint32_t* exited;            // CTAs of this launch that have left
     float* accept_prob;
     float b_out;
     uint32_t* status;
@@ -301,8 +301,6 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * C::STAGES + 4);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    if (blockIdx.x == gridDim.x - 1)
-        for (int i = tid; i < P.ready_words; i += HEAD_THREADS) P.ready_next[i] = 0;
     constexpr int TM = PAIR ? 2 * BM : BM;                                // rows of a tile
     const uint32_t rank = PAIR ? pair_rank() : 0u;                        // 0: issues the pair's MMAs, owns its barriers
     const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;   // a CTA or a pair of CTAs
@@ -527,6 +525,19 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if constexpr (PAIR) pair_sync();      // nothing is in flight towards the other CTA's barriers or tensor memory any more
+    if (warp == 2) {                      // the CTA that leaves last puts the counters back to zero
+        uint32_t left = 0;
+        if (lane == 0) {
+            __threadfence();
+            left = atomicAdd(P.exited, 1u);
+        }
+        left = __shfl_sync(0xffffffffu, left, 0);
+        if (left == gridDim.x - 1) {
+            __threadfence();
+            for (int i = lane; i < P.depth * nrb; i += 32) P.ready[i] = 0;
+            if (lane == 0) *P.exited = 0;
+        }
+    }
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if constexpr (PAIR)
@@ -967,10 +978,8 @@ cudaError_t launch_chain_call(specdec_ctx* ctx, const __nv_bfloat16* x, const sp
     p.d = d;
     p.w_out = static_cast<const __nv_bfloat16*>(head->w_out);
     p.partial = ctx->head_partial;
-    const size_t set_words = (size_t)CHAIN_MAX * (((size_t)ctx->max_B * ctx->max_K + BM - 1) / BM + 1);
-    p.ready = ctx->head_ready + (size_t)ctx->head_ready_set * set_words;
-    p.ready_next = ctx->head_ready + (size_t)(ctx->head_ready_set ^ 1) * set_words;
-    p.ready_words = (int)set_words;
+    p.ready = ctx->head_ready + 1;
+    p.exited = ctx->head_ready;
     p.accept_prob = accept_prob;
     p.b_out = head->b_out;
     p.status = ctx->status;
@@ -992,7 +1001,6 @@ cudaError_t launch_chain_call(specdec_ctx* ctx, const __nv_bfloat16* x, const sp
             ctx->launches += 1;
         }
     }
-    ctx->head_ready_set ^= 1;                                  // the sets change roles only when something was launched
     return cudaSuccess;
 }
 

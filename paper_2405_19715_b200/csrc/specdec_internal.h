@@ -40,9 +40,8 @@ struct specdec_ctx {
     // acceptance-head activations (device, bf16) and split-N partial logits
     void* act[2] = {nullptr, nullptr};   // [max_B*max_K, max_d] each
     float* head_partial = nullptr;       // [max_B*max_K, max_d/32]
-    uint32_t* head_ready = nullptr;      // [2][8][ceil(max_B*max_K / 128) + 1] finished epilogue warps per (block, 128-row block); a call
-                                         // counts in one of the two sets and clears the other for the next call
-    int head_ready_set = 0;
+    uint32_t* head_ready = nullptr;      // [0]: CTAs of the head launch that have left; then [8][ceil(max_B*max_K / 128) + 1] finished
+                                         // epilogue warps per (block, 128-row block); all zero between launches (the kernel clears them)
     int head_pair = 1;                   // a pair of CTAs per 256-row tile (0: one CTA per 128-row tile)
     int head_coop = -1;                  // one cooperative launch for all blocks: 0 ruled out or refused (one launch per block)
     HeadMapEntry head_maps[32];          // round-robin cache, keyed by (pointer, rows, cols, box rows, box cols)

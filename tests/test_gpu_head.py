@@ -99,6 +99,34 @@ def test_head_launch_forms_agree(rows, d, depth):
         np.testing.assert_allclose(got, ref, rtol=1e-5, atol=0, err_msg=str(key))
     ctx.close()
 
+
+@pytest.mark.parametrize("rows", [(3, 20), (25, 31)], ids=["60rows", "775rows"])
+def test_head_call_replayed_from_a_graph(rows):
+    """One captured call replayed three times in a row gives the eager call's bits every time: whatever the
+    kernels count in the context's scratch is back to its initial state when a call ends."""
+    B, K = rows
+    d, depth = 512, 3
+    ctx = specdec.Context(B, K, max_d=d)
+    hidden, Ws, bs, w_out, b_out = _head_problem(1200 + B, B, K, d, depth, True, std=0.02)
+    th, tw = specdec.from_numpy(hidden), specdec.from_numpy(w_out)
+    tW = [specdec.from_numpy(w) for w in Ws]
+    tb = [specdec.from_numpy(b) for b in bs]
+    out = torch.empty(B, K, dtype=torch.float32, device="cuda")
+    specdec.specdec_accept_head(ctx, th, tW, tb, tw, b_out, out)
+    torch.cuda.synchronize()
+    want = out.clone()
+    s = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=s):
+        specdec.specdec_accept_head(ctx, th, tW, tb, tw, b_out, out)
+    for _ in range(3):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, want)
+    assert ctx.device_status() == 0
+    ctx.close()
+
 @pytest.mark.parametrize("rows", [1, 2, 3, 4, 5, 8, 9, 13, 16, 17, 32, 33, 64, 65])
 @pytest.mark.parametrize("d,depth,with_bias", [(256, 1, True), (512, 3, False), (4096, 2, True)])
 def test_head_few_rows(rows, d, depth, with_bias):
