@@ -92,27 +92,17 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t sr
                  ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
-// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled:
-// start address, leading offset 16 B (unused by swizzled layouts), 1024 B between 8-row groups,
-// descriptor version 1, layout type SWIZZLE_128B.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-    return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
-}
 // Instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, M = 128, N = BN.
 __host__ __device__ constexpr uint32_t umma_idesc(int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 }
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
-}
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled: start
+// address >> 4 in bits 0-13, leading offset 16 B (unused by swizzled layouts) in bit 16; in the high word
+// 1024 B between 8-row groups, descriptor version 1, layout type SWIZZLE_128B.
 // The four MMAs of one 64-wide k-block in one statement.  `a_lo`, `b_lo` are the low words of the operands'
-// descriptors at k = 0 (address >> 4 in bits 0-13, leading offset in bit 16); a step of 16 bf16 along K is 32
-// bytes, i.e. + 2 in that word, and the high word (stride, version, swizzle) is the same for every tile, so
-// the issuing thread spends one add per descriptor instead of rebuilding 64-bit values.  `acc_first` is the
+// descriptors at k = 0; a step of 16 bf16 along K is 32 bytes, i.e. + 2 in that word, and the high word is
+// the same for every tile, so the issuing thread spends one add per descriptor instead of rebuilding 64-bit
+// values.  `acc_first` is the
 // accumulate flag of the first MMA (0 on a tile's first k-block); the other three always accumulate.
 constexpr uint32_t UMMA_DESC_HI = 64u | (1u << 14) | (2u << 29);
 __device__ __forceinline__ uint32_t umma_desc_lo(uint32_t smem_addr) { return ((smem_addr >> 4) & 0x3FFFu) | (1u << 16); }
@@ -211,13 +201,11 @@ __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w &
 
 struct BlockParams {
     const __nv_bfloat16* X;      // [M, d] input of the block (also the residual)
-    const __nv_bfloat16* W;      // [d, d] weights, (out, in)
     const __nv_bfloat16* bias;   // [d] or null
     __nv_bfloat16* Y;            // [M, d] output, null for the last block
     const __nv_bfloat16* w_out;  // [d], last block only
     float* partial;              // [M, 2 * d / BN], last block only
     int M, d;
-    int sm_count;
     uint32_t* status;
     // weights-as-M kernel, last block: the CTA that finishes last adds the partial dots and applies the sigmoid
     int32_t* done_ctr;
@@ -671,10 +659,8 @@ head_swap_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant
                 mbar_wait(full0 + 8 * stage, phase, budget);
                 if (kb == 0) HEAD_STAMP(2);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a = base + stage * stage_bytes, b = a + a_bytes;
-#pragma unroll
-                for (int k = 0; k < BK / UMMA_K; ++k)
-                    umma_bf16(tmem, umma_desc(a + k * UMMA_K * 2), umma_desc(b + k * UMMA_K * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+                const uint32_t a_lo = umma_desc_lo(base + stage * stage_bytes);
+                umma_kblock(tmem, a_lo, a_lo + (a_bytes >> 4), idesc, kb != 0 ? 1u : 0u);
                 umma_commit(empty0 + 8 * stage);
                 if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
             }
@@ -1064,14 +1050,12 @@ extern "C" int specdec_accept_head(specdec_ctx* ctx, const void* hidden, const s
                 return fail(ctx, SPECDEC_ECUDA, "accept_head: cuTensorMapEncodeTiled failed");
             BlockParams p;
             p.X = x;
-            p.W = static_cast<const __nv_bfloat16*>(head->W[k]);
             p.bias = static_cast<const __nv_bfloat16*>(head->b ? head->b[k] : nullptr);
             p.Y = last ? nullptr : static_cast<__nv_bfloat16*>(ctx->act[k & 1]);
             p.w_out = last ? static_cast<const __nv_bfloat16*>(head->w_out) : nullptr;
             p.partial = last ? ctx->head_partial : nullptr;
             p.M = (int)M;
             p.d = d;
-            p.sm_count = ctx->sm_count;
             p.status = ctx->status;
             p.done_ctr = ctx->task_ctl + 6;
             p.accept_prob = accept_prob;
