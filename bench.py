@@ -745,9 +745,10 @@ def run_head_phases(args):
             warnings.simplefilter("ignore", RuntimeWarning)
             a = np.nanmedian(np.stack(tl), 0)
             cyc = np.nanmedian(np.stack(cy), 0)
-        print(f"acceptance head, M={M} rows, d={d}, D={D}: tiles of the call's launch (both blocks: tile g of the launch is tile "
-              f"g mod 512 of block g div 512 at M=4096) on its first and its last CTA; microseconds from the launch's first "
-              f"stamp, median of {len(tl)} isolated calls; whole call by CUDA events {1e3 * np.mean(ms):.1f} us")
+        print(f"acceptance head, M={M} rows, d={d}, D={D}: tiles of the call's launch (all blocks: a CTA's tiles in the order it "
+              f"works on them, first block first) on its first and its last CTA (a pair's MMA-side stamps are its even CTA's: "
+              f"the last CTA of a paired launch has no row); microseconds from the launch's first stamp, median of {len(tl)} "
+              f"isolated calls; whole call by CUDA events {1e3 * np.mean(ms):.1f} us")
         print("| CTA | tile | first k-block requested | accumulator free | first k-block landed | all MMAs issued | accumulator complete | epilogue done | main loop (landed to issued), SM cycles | SM MHz in it |\n|---|---|---|---|---|---|---|---|---|---|")
         f = lambda v: "-" if np.isnan(v) else f"{v:.2f}"
         for c in range(2):
