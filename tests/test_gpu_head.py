@@ -52,14 +52,15 @@ def test_head_small_shapes(d, depth, with_bias, rows):
 
 
 @pytest.mark.parametrize("rows,d,depth", [((13, 47), 256, 1), ((13, 47), 512, 2), ((25, 31), 768, 2), ((64, 16), 1024, 3),
-                                          ((30, 20), 512, 8), ((75, 40), 768, 4), ((50, 42), 1024, 5)],
-                         ids=["611x256", "611x512", "775x768", "1024x1024", "600x512x8", "3000x768x4", "2100x1024x5"])
+                                          ((30, 20), 512, 8), ((80, 42), 768, 4), ((60, 42), 1024, 5)],
+                         ids=["611x256", "611x512", "775x768", "1024x1024", "600x512x8", "3360x768x4", "2520x1024x5"])
 def test_head_many_row_tiles(rows, d, depth):
     """Several row tiles with a ragged last one, widths up to 1024 and depth up to 8.  All blocks of a call are
-    tiles of one launch, a block's tiles waiting for the row block they read: the last two cases have 288 and
-    340 tiles, so every CTA gets two or three of them, from different blocks (the double-buffered accumulator
-    and the stage ring across tiles and blocks); depth 4 and more re-use the two activation buffers within
-    the launch.  The call is repeatable bit for bit."""
+    tiles of one launch, a block's tiles waiting for the row block they read: the last two cases have 168 and
+    200 tiles of 256 x 256 (a pair of CTAs each; the smaller cases get 128-wide tiles), so every pair gets two or
+    three of them, from different blocks (the double-buffered accumulator and the stage ring across tiles and
+    blocks); depth 4 and more re-use the two activation buffers within the launch.  The call is repeatable bit
+    for bit."""
     B, K = rows
     ctx = specdec.Context(B, K, max_d=d)
     hidden, Ws, bs, w_out, b_out = _head_problem(300 + d + depth, B, K, d, depth, True, std=0.02)
@@ -74,8 +75,8 @@ def test_head_many_row_tiles(rows, d, depth):
 
 
 
-@pytest.mark.parametrize("rows,d,depth", [((30, 20), 384, 3), ((75, 40), 768, 4), ((9, 33), 512, 2)],
-                         ids=["600x384x3", "3000x768x4", "297x512x2"])
+@pytest.mark.parametrize("rows,d,depth", [((30, 20), 384, 3), ((80, 42), 768, 4), ((9, 33), 512, 2)],
+                         ids=["600x384x3", "3360x768x4", "297x512x2"])
 def test_head_launch_forms_agree(rows, d, depth):
     """The three forms specdec_accept_head falls back through for more than 256 rows -- pairs of CTAs in one
     cooperative launch, one CTA per tile in one cooperative launch, one launch per block (with and without
