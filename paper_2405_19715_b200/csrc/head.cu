@@ -144,7 +144,7 @@ __device__ __forceinline__ uint32_t pair_map(uint32_t a, uint32_t rank) {
     return r;
 }
 // TMA load by one CTA of a pair whose bytes are counted on the EVEN CTA's barrier (peer bit of the barrier's
-// cluster address cleared).  No multicast: each CTA fetches its own operands.
+// cluster address cleared).  Each CTA fetches its own operands.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
