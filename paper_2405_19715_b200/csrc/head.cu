@@ -266,13 +266,14 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
 }
 
 // Persistent over the tiles of all its blocks: tile g = (block, row block, column tile), column tile fastest,
-// block slowest; CTA c works on tiles c, c + grid, ...  A tile of block l > first reads rows that the 128-row
-// tiles of block l - 1 in the same row block wrote, so its TMA thread first waits until `ready` shows all of
-// them finished (every epilogue warp counts once per tile, after its stores).  Those tiles come earlier in the
-// order, so with all CTAs resident (the launch is cooperative) the tile with the lowest unfinished index never
-// waits for an unfinished one; the wait is bounded all the same.  With 512 tiles per block on 148 SMs two blocks
-// take 7 rounds in one launch instead of 4 + 4 in two, and only the first tile of the launch waits for its
-// operands with nothing to overlap.  The accumulator is double-buffered in tensor memory (2 x BN columns), so
+// block slowest; worker w (a CTA, or with PAIR a cluster of two CTAs that share a 256-row tile, each loading
+// and finishing its own 128 rows) works on tiles w, w + workers, ...  A CTA's part of a tile of block l > first
+// reads 128 rows that the tiles of block l - 1 in the same row block wrote, so its TMA thread first waits until
+// `ready` shows all of them finished (every epilogue warp counts once per tile, after its stores).  Those tiles
+// come earlier in the order, so with all CTAs resident (the launch is cooperative) the tile with the lowest
+// unfinished index never waits for an unfinished one; the wait is bounded all the same.  With 512 tiles per
+// block on 148 SMs two blocks take 7 rounds in one launch instead of 4 + 4 in two, and only the first tile of
+// the launch waits for its operands with nothing to overlap.  The accumulator is double-buffered in tensor memory (2 x BN columns), so
 // the epilogue of one tile runs while the MMAs of the next are issued.  In the head's last block the warp that
 // completes a row block's count adds the block's partial dots in column order and applies the sigmoid.
 template <int BN, bool PAIR>
