@@ -334,6 +334,7 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             uint32_t stage = 0, phase = 0, it = 0;
+            bool wrapped = false;                              // the ring has been gone round at least once
             for (int g = worker; g < ntiles; g += nworkers, ++it) {
                 const int l = P.first + g / per_block, t = g % per_block;
                 const int m0 = (t / ntn) * TM + (int)rank * BM;                         // this CTA's rows of X
@@ -370,8 +371,17 @@ head_chain_kernel(const __grid_constant__ ChainParams P) {
                             tma_load_2d(b, mw, k0, n0, full0 + 8 * stage);
                         }
                     }
-                    if (++stage == C::STAGES) { stage = 0; phase ^= 1u; }
+                    if (++stage == C::STAGES) { stage = 0; phase ^= 1u; wrapped = true; }
                 }
+            }
+            // Before this CTA may end, every copy it asked for has landed and been consumed: each stage's last
+            // load (on the CTA that owns the full barrier) and the MMAs that read it.  All of it has happened
+            // long ago unless a wait gave up, in which case these waits are short as well.
+            for (uint32_t s = 0; s < (uint32_t)C::STAGES; ++s) {
+                if (s >= stage && !wrapped) continue;           // never used
+                const uint32_t ph = s < stage ? phase : phase ^ 1u;
+                if (rank == 0) mbar_wait(full0 + 8 * s, ph, budget);
+                mbar_wait(empty0 + 8 * s, ph, budget);
             }
         }
     } else if (warp == 1) {
